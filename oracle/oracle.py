@@ -1,0 +1,97 @@
+"""ctypes front for the plain C++ oracle in infaas_oracle.cpp.
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  It holds the per-variant load state (`queued`,
+`served_total`, counters) as numpy arrays and passes plain pointers to the C++ code,
+which is where every formula lives (Section 4.1 "Case I" selection, the cost objective
+of Section 2.2, the load bookkeeping of Section 4.2.2).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "infaas_oracle.cpp")
+_LIB = os.path.join(_HERE, "libinfaas_oracle.so")
+_lib = None
+
+NO_FEASIBLE_BIT = 0x80000000
+INVALID = 0xFFFFFFFF
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with the host compiler (-O2, no tuning flags)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread",
+                               _SRC, "-o", tmp])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.oracle_pred_lat.restype = ctypes.c_uint32
+        lib.oracle_pred_lat.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint16]
+        lib.oracle_select.restype = None
+        lib.oracle_select.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
+                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p,
+                                      ctypes.c_int]
+        lib.oracle_load_update.restype = None
+        lib.oracle_load_update.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                           ctypes.c_uint64, ctypes.c_uint32]
+        _lib = lib
+    return _lib
+
+
+def pred_lat(lat_us: int, queued: int, batch: int) -> int:
+    return int(_load().oracle_pred_lat(lat_us, queued, batch))
+
+
+def _ptr(a: np.ndarray) -> int:
+    assert a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data
+
+
+class OracleCatalog:
+    """Catalog rows + load state; `select` and `load_update` mirror the library's calls."""
+
+    def __init__(self, rows: np.ndarray, n_tasks: int):
+        assert rows.dtype.itemsize == 24
+        self.rows = np.ascontiguousarray(rows).copy()
+        self.n_tasks = int(n_tasks)
+        self.n_variants = int(rows.shape[0])
+        self.queued = self.rows["queued"].astype(np.uint32).copy()
+        self.served_total = np.zeros(self.n_variants, np.uint64)
+        self.counters = np.zeros(3, np.uint64)
+
+    def pred_lat(self) -> np.ndarray:
+        r = self.rows
+        return np.array([pred_lat(int(r["lat_us"][v]), int(self.queued[v]), int(r["batch"][v]))
+                         for v in range(self.n_variants)], np.uint32)
+
+    def select(self, task, slo_us, min_acc_bp, n_threads: int = 1) -> np.ndarray:
+        task = np.ascontiguousarray(task, np.uint16)
+        slo_us = np.ascontiguousarray(slo_us, np.uint32)
+        min_acc_bp = np.ascontiguousarray(min_acc_bp, np.uint16)
+        n = task.shape[0]
+        assert slo_us.shape[0] == n and min_acc_bp.shape[0] == n
+        out = np.empty(n, np.uint32)
+        _load().oracle_select(_ptr(self.rows), self.n_variants, self.n_tasks, _ptr(self.queued),
+                              _ptr(task), _ptr(slo_us), _ptr(min_acc_bp), n, _ptr(out),
+                              int(n_threads))
+        return out
+
+    def load_update(self, decision, window_us: int) -> None:
+        decision = np.ascontiguousarray(decision, np.uint32)
+        _load().oracle_load_update(_ptr(self.rows), self.n_variants, _ptr(self.queued),
+                                   _ptr(self.served_total), _ptr(self.counters),
+                                   _ptr(decision), decision.shape[0], int(window_us))
