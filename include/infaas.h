@@ -1,0 +1,149 @@
+/* infaas.h -- C ABI of the batched model-variant selection library (CUDA, sm_100a).
+ *
+ * The library answers, for a batch of queries, the question the paper's dispatcher asks on
+ * the arrival of every query (Section 4.1, "Case I"): which profiled model-variant of the
+ * query's application should serve it, given a latency requirement and an accuracy
+ * requirement (Section 3.1, Table 4).  Between batches it folds the decisions back into
+ * per-variant load (Section 4.2.2) so that the next batch sees load-adjusted latencies
+ * (Section 4, the list of dynamic aspects a static profile misses).
+ *
+ * Units: latency in microseconds (u32), accuracy in basis points (u16, 0..10000), cost in
+ * integer units (u32).  All arithmetic is unsigned integer arithmetic; results are exact.
+ *
+ * Every function returns 0 on success or a negative INFAAS_E_* code.  No function throws,
+ * aborts, or makes the GPU fault on bad *values* inside the query arrays.
+ */
+#ifndef INFAAS_H_
+#define INFAAS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct infaas_catalog infaas_catalog; /* opaque; owns all catalog device memory */
+
+/* One profiled model-variant (Section 2.1 lists what defines a variant; Section 3.2,
+ * "Variant-Generator and Variant-Profiler", lists what is recorded for it).  The variant
+ * id is the row's index in the array given to infaas_catalog_load. */
+typedef struct {
+  uint16_t task;     /* application / task index, < n_tasks                              */
+  uint16_t arch;     /* model architecture code (carried, not used by selection)         */
+  uint8_t hw;        /* hardware platform code   (carried, not used by selection)        */
+  uint8_t opt;       /* framework / graph-optimiser code (carried, not used)             */
+  uint16_t batch;    /* batch size the variant is optimised for, >= 1                    */
+  uint32_t lat_us;   /* profiled latency of one batch, microseconds, >= 1                */
+  uint16_t acc_bp;   /* accuracy, basis points, 0..10000                                 */
+  uint16_t reserved; /* must be 0                                                        */
+  uint32_t cost;     /* cost, integer units                                              */
+  uint32_t queued;   /* queries already queued on this variant (initial load snapshot)   */
+} infaas_variant;    /* 24 bytes */
+
+/* Decision encoding (one u32 per query):
+ *   0 .. 2^31-2          id of the chosen variant (it meets both requirements)
+ *   bit 31 set           no variant meets the requirements; low 31 bits = nearest miss
+ *   0xFFFFFFFF           invalid query: task >= n_tasks or the task has no variant      */
+#define INFAAS_NO_FEASIBLE 0x80000000u
+#define INFAAS_INVALID 0xFFFFFFFFu
+
+#define INFAAS_OK 0
+#define INFAAS_E_NULL (-1)      /* a required pointer is NULL                             */
+#define INFAAS_E_BAD_TASK (-2)  /* a row's task >= n_tasks, or n_tasks == 0 / > 65535     */
+#define INFAAS_E_BAD_BATCH (-3) /* a row's batch == 0                                     */
+#define INFAAS_E_BAD_LAT (-4)   /* a row's lat_us == 0                                    */
+#define INFAAS_E_BAD_ACC (-5)   /* a row's acc_bp > 10000 or reserved != 0                */
+#define INFAAS_E_TOO_LARGE (-6) /* a size limit is exceeded (see each function)           */
+#define INFAAS_E_CUDA (-7)      /* a CUDA call failed; infaas_last_cuda_error() has text  */
+#define INFAAS_E_ALIGN (-8)     /* a device array is not 16-byte aligned                  */
+#define INFAAS_E_DEVICE (-9)    /* a kernel reported an internal error (a bounded wait ran
+                                   out); the catalog is unchanged by that call            */
+
+/* Limits. */
+#define INFAAS_MAX_VARIANTS 0x7FFFFFFEu   /* ids must fit below bit 31                     */
+#define INFAAS_MAX_TASK_VARIANTS 8192u    /* variants of one task (sorted in shared memory) */
+
+/* Build the device catalog (Section 3.2, "Metadata Store": static profiles plus dynamic
+ * load, organised for fast lookup).  Validates the rows, buckets them by task, uploads
+ * them as a struct of arrays, computes each variant's load-adjusted latency
+ *     pred_lat = min(2^32-1, lat_us + floor(queued * lat_us / batch))
+ * and builds, per task, the list of non-dominated variants in (cost, pred_lat, -acc, id)
+ * order that the selection kernel scans.
+ *   rows         HOST pointer, n_variants rows, copied; the caller keeps ownership.
+ *   n_variants   1 .. INFAAS_MAX_VARIANTS; at most INFAAS_MAX_TASK_VARIANTS per task.
+ *   n_tasks      1 .. 65535.  Tasks without rows are allowed (their queries are INVALID).
+ *   cuda_device  device ordinal; all later calls on this catalog run on it.
+ *   out          receives the handle; release it with infaas_catalog_free.
+ * Allocates device memory and synchronises the device.  Errors: E_NULL, E_BAD_*,
+ * E_TOO_LARGE, E_CUDA.  On error *out is NULL and nothing is leaked. */
+int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_t n_tasks,
+                        int cuda_device, infaas_catalog **out);
+
+/* Decide n queries against the catalog's current load snapshot (Section 4.1, Case I; the
+ * cost objective is the one of Section 2.2's worked example around Table 2).
+ * For query q over the variants v of task d_task[q]:
+ *     feasible(v)  <=>  pred_lat(v) <= d_slo_us[q]  and  acc_bp(v) >= d_min_acc_bp[q]
+ *   - some v feasible: d_decision[q] = the feasible v smallest in (cost, pred_lat,
+ *     10000-acc_bp, id), lexicographically;
+ *   - none feasible (Section 4.1: suggest the closest variant): with
+ *     d(v) = 10000*max(0, pred_lat-slo) + slo*max(0, min_acc-acc_bp)  (64-bit),
+ *     d_decision[q] = INFAAS_NO_FEASIBLE | the v smallest in (d, cost, pred_lat,
+ *     10000-acc_bp, id);
+ *   - task out of range or without variants: INFAAS_INVALID.
+ * All queries of one call see the same snapshot.
+ *   d_task, d_slo_us, d_min_acc_bp   DEVICE arrays of n elements, 16-byte aligned, read only.
+ *   d_decision                       DEVICE array of n u32, 16-byte aligned, written.
+ *   cuda_stream                      a cudaStream_t (NULL = default stream).
+ * Asynchronous and stream-ordered; allocates nothing.  n == 0 is a successful no-op.
+ * Errors: E_NULL, E_ALIGN, E_CUDA (launch failure).  A kernel-internal error is reported by
+ * the next infaas_catalog_get_state as E_DEVICE. */
+int infaas_select_batch(infaas_catalog *c, const uint16_t *d_task, const uint32_t *d_slo_us,
+                        const uint16_t *d_min_acc_bp, uint64_t n, uint32_t *d_decision,
+                        void *cuda_stream);
+
+/* Close a window (Section 4.2.2: load per variant from the queries it serves and its batch
+ * size; Section 5: load statistics are refreshed periodically).  Tallies the window's
+ * decisions per variant, advances every variant's queue by one window and rebuilds the
+ * load-adjusted latencies and the per-task scan lists:
+ *     count(v)   = #{q : d_decision[q] == v}          (bit 31 clear and v < n_variants)
+ *     drain(v)   = min(2^32-1, floor(window_us * batch / lat_us))
+ *     queued(v)  = max(0, min(2^32-1, queued + count) - drain)
+ *     served_total(v) += count(v)
+ * Decisions with bit 31 set add no load; INFAAS_INVALID and ids >= n_variants are counted
+ * as invalid and otherwise ignored.
+ *   d_decision   DEVICE array of n u32 (16-byte aligned), read only; n <= 2^32-1.
+ * Asynchronous, stream-ordered, allocates nothing; must be ordered (same stream or an
+ * event) before the next infaas_select_batch that should see the new load.
+ * Errors: E_NULL, E_ALIGN, E_TOO_LARGE, E_CUDA. */
+int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n,
+                       uint32_t window_us, void *cuda_stream);
+
+/* Copy the load state to HOST arrays (any of the four may be NULL to skip it):
+ *   h_queued[n_variants], h_pred_lat_us[n_variants], h_served_total[n_variants] indexed by
+ *   variant id; h_counters[3] = feasible decisions tallied, NO_FEASIBLE decisions seen,
+ *   invalid decisions seen, summed over all infaas_load_update calls.
+ * Synchronises cuda_stream.  Returns E_DEVICE if any kernel of this catalog recorded an
+ * internal error since the last call. */
+int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_pred_lat_us,
+                             uint64_t *h_served_total, uint64_t h_counters[3],
+                             void *cuda_stream);
+
+/* Copy one task's scan list to HOST: the ids of its non-dominated variants in scan order.
+ * h_ids may be NULL to query the length only; at most `cap` ids are written.
+ * *h_len receives the list's length.  Synchronises cuda_stream.  For inspection/tests. */
+int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_ids,
+                                uint32_t cap, uint32_t *h_len, void *cuda_stream);
+
+/* Release the catalog and its device memory.  NULL is allowed. */
+void infaas_catalog_free(infaas_catalog *c);
+
+/* Text for an INFAAS_E_* code; never NULL. */
+const char *infaas_strerror(int code);
+
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char *infaas_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* INFAAS_H_ */

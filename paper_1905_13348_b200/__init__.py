@@ -1,0 +1,17 @@
+"""Batched model-variant selection and load tallies on B200 (C-ABI CUDA library + binding).
+
+`workloads` (input generators) imports without the CUDA library; the binding's functions
+are resolved lazily and raise if the library has not been built.
+"""
+from . import workloads  # noqa: F401
+
+_BINDING = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
+            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "Catalog", "InfaasError",
+            "NO_FEASIBLE", "INVALID")
+
+
+def __getattr__(name):
+    if name in _BINDING:
+        from . import binding
+        return getattr(binding, name)
+    raise AttributeError(name)

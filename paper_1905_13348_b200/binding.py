@@ -1,0 +1,147 @@
+"""Thin ctypes binding of the C ABI in include/infaas.h (argument marshalling only).
+
+Every step of the path runs inside the CUDA library; this module passes pointers and
+sizes.  Device arrays are torch CUDA tensors (torch is used for device memory and streams
+only).  There is no CPU fallback: if the library has not been built, importing the symbols
+raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+from .build import LIB_PATH
+
+NO_FEASIBLE = 0x80000000
+INVALID = 0xFFFFFFFF
+
+_lib = None
+
+EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
+           "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
+           "infaas_strerror", "infaas_last_cuda_error")
+
+
+class InfaasError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        lib = _load()
+        msg = lib.infaas_strerror(code).decode()
+        cuda = lib.infaas_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({code})" + (f" [{cuda}]" if code == -7 and cuda else ""))
+        self.code = code
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"CUDA library not built: {LIB_PATH} is missing "
+                           "(run `python -m paper_1905_13348_b200.build`); there is no fallback")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, u32, u64, i32 = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int
+    lib.infaas_catalog_load.argtypes = [vp, u32, u32, i32, ctypes.POINTER(vp)]
+    lib.infaas_select_batch.argtypes = [vp, vp, vp, vp, u64, vp, vp]
+    lib.infaas_load_update.argtypes = [vp, vp, u64, u32, vp]
+    lib.infaas_catalog_get_state.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.infaas_catalog_get_frontier.argtypes = [vp, u32, vp, u32, ctypes.POINTER(u32), vp]
+    lib.infaas_catalog_free.argtypes = [vp]
+    lib.infaas_catalog_free.restype = None
+    for name in ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
+                 "infaas_catalog_get_state", "infaas_catalog_get_frontier"):
+        getattr(lib, name).restype = i32
+    lib.infaas_strerror.argtypes = [i32]
+    lib.infaas_strerror.restype = ctypes.c_char_p
+    lib.infaas_last_cuda_error.argtypes = []
+    lib.infaas_last_cuda_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(code: int, where: str) -> None:
+    if code != 0:
+        raise InfaasError(code, where)
+
+
+def _dev_ptr(t, dtype_name: str):
+    """Device pointer of a contiguous torch CUDA tensor of the given integer width."""
+    import torch
+    widths = {"u16": (torch.int16, torch.uint16), "u32": (torch.int32, torch.uint32)}
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous() or t.dtype not in widths[dtype_name]:
+        raise TypeError(f"expected a contiguous CUDA tensor of {dtype_name}, got {t.dtype} on {t.device}")
+    return t.data_ptr()
+
+
+def _stream_ptr(stream):
+    import torch
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class Catalog:
+    """Owner of an `infaas_catalog*` handle."""
+
+    def __init__(self, handle: int, n_variants: int, n_tasks: int, device: int):
+        self.handle = ctypes.c_void_p(handle)
+        self.n_variants, self.n_tasks, self.device = n_variants, n_tasks, device
+
+    def free(self) -> None:
+        if self.handle:
+            _load().infaas_catalog_free(self.handle)
+            self.handle = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def infaas_catalog_load(rows: np.ndarray, n_tasks: int, cuda_device: int = 0) -> Catalog:
+    """rows: host numpy array of 24-byte catalog rows (variant id = index)."""
+    rows = np.ascontiguousarray(rows)
+    if rows.dtype.itemsize != 24:
+        raise TypeError("rows must be an array of 24-byte catalog rows")
+    out = ctypes.c_void_p(None)
+    _check(_load().infaas_catalog_load(rows.ctypes.data, rows.shape[0], n_tasks, cuda_device,
+                                       ctypes.byref(out)), "infaas_catalog_load")
+    return Catalog(out.value, int(rows.shape[0]), int(n_tasks), int(cuda_device))
+
+
+def infaas_select_batch(cat: Catalog, d_task, d_slo_us, d_min_acc_bp, d_decision, n=None,
+                        stream=None) -> None:
+    n = int(d_task.shape[0]) if n is None else int(n)
+    _check(_load().infaas_select_batch(cat.handle, _dev_ptr(d_task, "u16"), _dev_ptr(d_slo_us, "u32"),
+                                       _dev_ptr(d_min_acc_bp, "u16"), n, _dev_ptr(d_decision, "u32"),
+                                       _stream_ptr(stream)), "infaas_select_batch")
+
+
+def infaas_load_update(cat: Catalog, d_decision, window_us: int, n=None, stream=None) -> None:
+    n = int(d_decision.shape[0]) if n is None else int(n)
+    _check(_load().infaas_load_update(cat.handle, _dev_ptr(d_decision, "u32"), n, int(window_us),
+                                      _stream_ptr(stream)), "infaas_load_update")
+
+
+def infaas_catalog_get_state(cat: Catalog, stream=None) -> dict:
+    queued = np.empty(cat.n_variants, np.uint32)
+    pred = np.empty(cat.n_variants, np.uint32)
+    served = np.empty(cat.n_variants, np.uint64)
+    counters = np.zeros(3, np.uint64)
+    _check(_load().infaas_catalog_get_state(cat.handle, queued.ctypes.data, pred.ctypes.data,
+                                            served.ctypes.data, counters.ctypes.data,
+                                            _stream_ptr(stream)), "infaas_catalog_get_state")
+    return {"queued": queued, "pred_lat_us": pred, "served_total": served, "counters": counters}
+
+
+def infaas_catalog_get_frontier(cat: Catalog, task: int, stream=None) -> np.ndarray:
+    ids = np.empty(max(1, cat.n_variants), np.uint32)
+    ln = ctypes.c_uint32(0)
+    _check(_load().infaas_catalog_get_frontier(cat.handle, int(task), ids.ctypes.data, ids.shape[0],
+                                               ctypes.byref(ln), _stream_ptr(stream)),
+           "infaas_catalog_get_frontier")
+    return ids[:ln.value].copy()

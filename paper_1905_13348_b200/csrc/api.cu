@@ -1,0 +1,326 @@
+// C ABI of the library (declared in include/infaas.h): handle management, validation,
+// the host side of the catalog packer, and the calls that launch the kernels.
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+using infaas::DeviceCatalog;
+
+struct infaas_catalog {
+  int device = 0;
+  int sm_count = 0;
+  DeviceCatalog d{};
+  void *arena = nullptr;                 // one device allocation holds every array
+  std::vector<uint32_t> slot_of_id;      // host copy, for get_state
+  std::vector<uint32_t> task_off, reg_off;
+  uint32_t select_smem = 0;              // dynamic shared memory given to the selection kernel
+  uint32_t worst_blob_bytes = 0;         // image size if no variant were dominated
+};
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int cuda_fail(cudaError_t e) {
+  g_cuda_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e);
+  (void)cudaGetLastError();   // clear the sticky-free error state
+  return INFAAS_E_CUDA;
+}
+
+#define CUDA_TRY(expr)                         \
+  do {                                         \
+    cudaError_t e__ = (expr);                  \
+    if (e__ != cudaSuccess) return cuda_fail(e__); \
+  } while (0)
+
+// Makes the catalog's device current for the scope of one call.
+struct DeviceScope {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t status = cudaSuccess;
+  explicit DeviceScope(int dev) {
+    status = cudaGetDevice(&prev);
+    if (status == cudaSuccess && prev != dev) {
+      status = cudaSetDevice(dev);
+      switched = status == cudaSuccess;
+    }
+  }
+  ~DeviceScope() {
+    if (switched) (void)cudaSetDevice(prev);
+  }
+};
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Re-reads the image size from the device and sizes the selection kernel's shared memory
+// with headroom for growth between two such refreshes.
+int refresh_select_plan(infaas_catalog *c, cudaStream_t stream) {
+  uint32_t hdr[4] = {0, 0, 0, 0};
+  CUDA_TRY(cudaMemcpyAsync(hdr, c->d.blob_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, stream));
+  CUDA_TRY(cudaStreamSynchronize(stream));
+  uint64_t want = (uint64_t)hdr[0] + hdr[0] / 2 + 4096;
+  if (want > c->worst_blob_bytes) want = c->worst_blob_bytes;
+  if (want > infaas::SELECT_MAX_SMEM) want = infaas::SELECT_MAX_SMEM;
+  c->select_smem = (uint32_t)(want & ~(uint64_t)15);
+  return INFAAS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *infaas_strerror(int code) {
+  switch (code) {
+    case INFAAS_OK: return "ok";
+    case INFAAS_E_NULL: return "a required pointer is NULL";
+    case INFAAS_E_BAD_TASK: return "row task out of range, or n_tasks is 0 or above 65535";
+    case INFAAS_E_BAD_BATCH: return "row batch size is 0";
+    case INFAAS_E_BAD_LAT: return "row latency is 0";
+    case INFAAS_E_BAD_ACC: return "row accuracy above 10000 basis points, or reserved field not 0";
+    case INFAAS_E_TOO_LARGE: return "size limit exceeded";
+    case INFAAS_E_CUDA: return "CUDA call failed (see infaas_last_cuda_error)";
+    case INFAAS_E_ALIGN: return "device array is not 16-byte aligned";
+    case INFAAS_E_DEVICE: return "a kernel reported an internal error";
+    default: return "unknown error code";
+  }
+}
+
+const char *infaas_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_t n_tasks,
+                        int cuda_device, infaas_catalog **out) {
+  if (out) *out = nullptr;
+  if (!rows || !out) return INFAAS_E_NULL;
+  if (n_tasks == 0 || n_tasks > 65535u) return INFAAS_E_BAD_TASK;
+  if (n_variants == 0 || n_variants > INFAAS_MAX_VARIANTS) return INFAAS_E_TOO_LARGE;
+
+  // ---- validate and bucket by task (stable: ascending id inside a task) ----
+  std::vector<uint32_t> task_off(n_tasks + 1, 0);
+  for (uint32_t v = 0; v < n_variants; ++v) {
+    const infaas_variant &r = rows[v];
+    if (r.task >= n_tasks) return INFAAS_E_BAD_TASK;
+    if (r.batch == 0) return INFAAS_E_BAD_BATCH;
+    if (r.lat_us == 0) return INFAAS_E_BAD_LAT;
+    if (r.acc_bp > 10000 || r.reserved != 0) return INFAAS_E_BAD_ACC;
+    task_off[r.task + 1]++;
+  }
+  uint32_t max_task = 0;
+  for (uint32_t t = 0; t < n_tasks; ++t) {
+    if (task_off[t + 1] > max_task) max_task = task_off[t + 1];
+    task_off[t + 1] += task_off[t];
+  }
+  if (max_task > INFAAS_MAX_TASK_VARIANTS) return INFAAS_E_TOO_LARGE;
+  std::vector<uint32_t> reg_off(n_tasks + 1, 0);
+  for (uint32_t t = 0; t < n_tasks; ++t)
+    reg_off[t + 1] = reg_off[t] + (uint32_t)round_up(task_off[t + 1] - task_off[t], 4);
+  const uint32_t region_entries = reg_off[n_tasks];
+
+  std::vector<uint32_t> h_lat(n_variants), h_cost(n_variants), h_id(n_variants), h_queued(n_variants),
+      slot_of_id(n_variants);
+  std::vector<uint16_t> h_batch(n_variants), h_acc(n_variants);
+  {
+    std::vector<uint32_t> cursor(task_off.begin(), task_off.end() - 1);
+    for (uint32_t v = 0; v < n_variants; ++v) {
+      const infaas_variant &r = rows[v];
+      const uint32_t s = cursor[r.task]++;
+      h_lat[s] = r.lat_us; h_batch[s] = r.batch; h_acc[s] = r.acc_bp; h_cost[s] = r.cost;
+      h_id[s] = v; h_queued[s] = r.queued; slot_of_id[v] = s;
+    }
+  }
+
+  infaas_catalog *c = new (std::nothrow) infaas_catalog();
+  if (!c) return INFAAS_E_TOO_LARGE;
+  c->device = cuda_device;
+  DeviceScope scope(cuda_device);
+  if (scope.status != cudaSuccess) { delete c; return cuda_fail(scope.status); }
+
+  // ---- one arena, carved into 256-byte aligned arrays ----
+  const uint32_t n_tasks_pad = (n_tasks + 1u) & ~1u;
+  const uint64_t worst_blob = (uint64_t)n_tasks_pad * 8u + (uint64_t)round_up(n_variants, 4) * 12u;
+  if (worst_blob > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
+  size_t total = 0;
+  auto carve = [&total](size_t bytes) { size_t off = total; total += round_up(bytes, 256); return off; };
+  const size_t o_task_off = carve((n_tasks + 1) * 4), o_reg_off = carve((n_tasks + 1) * 4);
+  const size_t o_lat = carve((size_t)n_variants * 4), o_batch = carve((size_t)n_variants * 2);
+  const size_t o_acc = carve((size_t)n_variants * 2), o_cost = carve((size_t)n_variants * 4);
+  const size_t o_id = carve((size_t)n_variants * 4), o_queued = carve((size_t)n_variants * 4);
+  const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
+  const size_t o_count = carve((size_t)n_variants * 4);
+  const size_t o_fkey = carve((size_t)region_entries * 8), o_fid = carve((size_t)region_entries * 4);
+  const size_t o_flen = carve((size_t)n_tasks * 4);
+  const size_t o_blob = carve((size_t)worst_blob), o_hdr = carve(16);
+  const size_t o_counters = carve(24), o_done = carve(4), o_err = carve(4);
+
+#define LOAD_TRY(expr)                                                     \
+  do {                                                                     \
+    cudaError_t e__ = (expr);                                              \
+    if (e__ != cudaSuccess) { infaas_catalog_free(c); return cuda_fail(e__); } \
+  } while (0)
+
+  cudaDeviceProp prop;
+  LOAD_TRY(cudaGetDeviceProperties(&prop, cuda_device));
+  c->sm_count = prop.multiProcessorCount;
+  LOAD_TRY(cudaMalloc(&c->arena, total));
+  unsigned char *base = static_cast<unsigned char *>(c->arena);
+  LOAD_TRY(cudaMemset(base, 0, total));
+  LOAD_TRY(cudaMemcpy(base + o_task_off, task_off.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_reg_off, reg_off.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_lat, h_lat.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_batch, h_batch.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_acc, h_acc.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_cost, h_cost.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_id, h_id.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_queued, h_queued.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
+
+  DeviceCatalog &d = c->d;
+  d.n_variants = n_variants;
+  d.n_tasks = n_tasks;
+  d.n_tasks_pad = n_tasks_pad;
+  d.max_task_variants = max_task;
+  d.region_entries = region_entries;
+  d.task_off = reinterpret_cast<const uint32_t *>(base + o_task_off);
+  d.reg_off = reinterpret_cast<const uint32_t *>(base + o_reg_off);
+  d.s_lat = reinterpret_cast<const uint32_t *>(base + o_lat);
+  d.s_batch = reinterpret_cast<const uint16_t *>(base + o_batch);
+  d.s_acc = reinterpret_cast<const uint16_t *>(base + o_acc);
+  d.s_cost = reinterpret_cast<const uint32_t *>(base + o_cost);
+  d.s_id = reinterpret_cast<const uint32_t *>(base + o_id);
+  d.s_queued = reinterpret_cast<uint32_t *>(base + o_queued);
+  d.s_pred = reinterpret_cast<uint32_t *>(base + o_pred);
+  d.s_served = reinterpret_cast<unsigned long long *>(base + o_served);
+  d.count_by_id = reinterpret_cast<uint32_t *>(base + o_count);
+  d.f_key = reinterpret_cast<unsigned long long *>(base + o_fkey);
+  d.f_id = reinterpret_cast<uint32_t *>(base + o_fid);
+  d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
+  d.blob = base + o_blob;
+  d.blob_capacity = (uint32_t)worst_blob;
+  d.blob_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
+  d.counters = reinterpret_cast<unsigned long long *>(base + o_counters);
+  d.done_ctr = reinterpret_cast<uint32_t *>(base + o_done);
+  d.err = reinterpret_cast<uint32_t *>(base + o_err);
+  c->slot_of_id.swap(slot_of_id);
+  c->task_off.swap(task_off);
+  c->reg_off.swap(reg_off);
+  c->worst_blob_bytes = (uint32_t)worst_blob;
+
+  LOAD_TRY(infaas::prepare_select_kernel());
+  LOAD_TRY(infaas::prepare_rebuild_kernel());
+  LOAD_TRY(infaas::launch_rebuild(d, /*advance_queues=*/false, 0, nullptr));
+  LOAD_TRY(cudaDeviceSynchronize());
+  int rc = refresh_select_plan(c, nullptr);
+  if (rc != INFAAS_OK) { infaas_catalog_free(c); return rc; }
+#undef LOAD_TRY
+  *out = c;
+  return INFAAS_OK;
+}
+
+int infaas_select_batch(infaas_catalog *c, const uint16_t *d_task, const uint32_t *d_slo_us,
+                        const uint16_t *d_min_acc_bp, uint64_t n, uint32_t *d_decision,
+                        void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  if (n == 0) return INFAAS_OK;
+  if (!d_task || !d_slo_us || !d_min_acc_bp || !d_decision) return INFAAS_E_NULL;
+  if (!aligned16(d_task) || !aligned16(d_slo_us) || !aligned16(d_min_acc_bp) || !aligned16(d_decision))
+    return INFAAS_E_ALIGN;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  CUDA_TRY(infaas::launch_select(c->d, d_task, d_slo_us, d_min_acc_bp, n, d_decision, c->sm_count,
+                                 c->select_smem, static_cast<cudaStream_t>(cuda_stream)));
+  return INFAAS_OK;
+}
+
+int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n,
+                       uint32_t window_us, void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  if (n > 0xFFFFFFFFull) return INFAAS_E_TOO_LARGE;
+  if (n > 0 && !d_decision) return INFAAS_E_NULL;
+  if (n > 0 && !aligned16(d_decision)) return INFAAS_E_ALIGN;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  CUDA_TRY(infaas::launch_tally(c->d, d_decision, n, s));
+  CUDA_TRY(infaas::launch_rebuild(c->d, /*advance_queues=*/true, window_us, s));
+  return INFAAS_OK;
+}
+
+int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_pred_lat_us,
+                             uint64_t *h_served_total, uint64_t h_counters[3], void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const uint32_t nv = c->d.n_variants;
+  std::vector<uint32_t> tmp32;
+  std::vector<unsigned long long> tmp64;
+  if (h_queued) {
+    tmp32.resize(nv);
+    CUDA_TRY(cudaMemcpyAsync(tmp32.data(), c->d.s_queued, (size_t)nv * 4, cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    for (uint32_t v = 0; v < nv; ++v) h_queued[v] = tmp32[c->slot_of_id[v]];
+  }
+  if (h_pred_lat_us) {
+    tmp32.resize(nv);
+    CUDA_TRY(cudaMemcpyAsync(tmp32.data(), c->d.s_pred, (size_t)nv * 4, cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    for (uint32_t v = 0; v < nv; ++v) h_pred_lat_us[v] = tmp32[c->slot_of_id[v]];
+  }
+  if (h_served_total) {
+    tmp64.resize(nv);
+    CUDA_TRY(cudaMemcpyAsync(tmp64.data(), c->d.s_served, (size_t)nv * 8, cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    for (uint32_t v = 0; v < nv; ++v) h_served_total[v] = tmp64[c->slot_of_id[v]];
+  }
+  if (h_counters) {
+    unsigned long long k[3];
+    CUDA_TRY(cudaMemcpyAsync(k, c->d.counters, sizeof(k), cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    for (int i = 0; i < 3; ++i) h_counters[i] = k[i];
+  }
+  uint32_t err = 0;
+  CUDA_TRY(cudaMemcpyAsync(&err, c->d.err, 4, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  int rc = refresh_select_plan(c, s);
+  if (rc != INFAAS_OK) return rc;
+  if (err != infaas::DEV_ERR_NONE) {
+    CUDA_TRY(cudaMemsetAsync(c->d.err, 0, 4, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+    return INFAAS_E_DEVICE;
+  }
+  return INFAAS_OK;
+}
+
+int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_ids, uint32_t cap,
+                                uint32_t *h_len, void *cuda_stream) {
+  if (!c || !h_len) return INFAAS_E_NULL;
+  if (task >= c->d.n_tasks) return INFAAS_E_BAD_TASK;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t len = 0;
+  CUDA_TRY(cudaMemcpyAsync(&len, c->d.f_len + task, 4, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  *h_len = len;
+  const uint32_t ncopy = len < cap ? len : cap;
+  if (h_ids && ncopy) {
+    CUDA_TRY(cudaMemcpyAsync(h_ids, c->d.f_id + c->reg_off[task], (size_t)ncopy * 4,
+                             cudaMemcpyDeviceToHost, s));
+    CUDA_TRY(cudaStreamSynchronize(s));
+  }
+  return INFAAS_OK;
+}
+
+void infaas_catalog_free(infaas_catalog *c) {
+  if (!c) return;
+  if (c->arena) {
+    DeviceScope scope(c->device);
+    (void)cudaFree(c->arena);
+  }
+  delete c;
+}
+
+}  // extern "C"

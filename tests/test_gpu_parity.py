@@ -1,0 +1,210 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, element by
+element on the same seeded inputs.  Integer work: the bar is bit-exact."""
+import numpy as np
+import pytest
+
+from oracle import OracleCatalog
+from paper_1905_13348_b200 import workloads as W
+from tests.helpers import INVALID, NO_FEASIBLE_BIT, rows_from
+
+pytestmark = pytest.mark.gpu
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def _to_dev(a):
+    torch = _torch()
+    view = {np.dtype("uint16"): np.int16, np.dtype("uint32"): np.int32}[a.dtype]
+    return torch.from_numpy(np.ascontiguousarray(a).view(view)).cuda()
+
+
+def _to_host_u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def gpu_select(cat, task, slo, acc):
+    import paper_1905_13348_b200 as P
+    torch = _torch()
+    d_task, d_slo, d_acc = _to_dev(task), _to_dev(slo), _to_dev(acc)
+    d_dec = torch.full((task.shape[0],), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    P.infaas_select_batch(cat, d_task, d_slo, d_acc, d_dec)
+    torch.cuda.synchronize()
+    return d_dec
+
+
+def assert_state_equal(cat, o):
+    import paper_1905_13348_b200 as P
+    st = P.infaas_catalog_get_state(cat)
+    assert np.array_equal(st["queued"], o.queued)
+    assert np.array_equal(st["pred_lat_us"], o.pred_lat())
+    assert np.array_equal(st["served_total"], o.served_total)
+    assert np.array_equal(st["counters"], o.counters)
+
+
+def run_both(w, n_threads=8, check_state=True):
+    """Whole workload through both sides; windowed if the workload says so."""
+    import paper_1905_13348_b200 as P
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    try:
+        if check_state:
+            assert_state_equal(cat, o)
+        step = w.window if w.window else max(1, w.n_queries)
+        for lo in range(0, w.n_queries, step):
+            s = slice(lo, min(w.n_queries, lo + step))
+            want = o.select(w.task[s], w.slo_us[s], w.min_acc_bp[s], n_threads)
+            d_dec = gpu_select(cat, w.task[s], w.slo_us[s], w.min_acc_bp[s])
+            got = _to_host_u32(d_dec)
+            bad = np.flatnonzero(got != want)
+            assert bad.size == 0, (w.name, lo, bad[:5], got[bad[:5]], want[bad[:5]])
+            if w.window:
+                P.infaas_load_update(cat, d_dec, w.window_us)
+                o.load_update(want, w.window_us)
+                if check_state:
+                    assert_state_equal(cat, o)
+        if not w.window:
+            P.infaas_load_update(cat, d_dec, 1000)
+            o.load_update(want, 1000)
+            assert_state_equal(cat, o)
+    finally:
+        cat.free()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("C1", {}),
+    ("C2", {"n_queries": 200_003}),
+    ("C3", {"n_queries": 12 * 8192 + 77, "window": 8192}),
+    ("C4", {"n_queries": 65_537}),
+    ("C5", {"n_windows": 6, "window": 4096}),
+])
+def test_configs_reduced(name, kw):
+    run_both(W.make(name, **kw))
+
+
+def test_heavy_load_windows_change_the_frontier():
+    # few queries' worth of drain per window: queues build up, scan lists change every window
+    w = W.make("C3", n_queries=20 * 4096, window=4096)
+    w.window_us = 300
+    run_both(w)
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 4, 5, 7, 8, 511, 2049])
+def test_ragged_sizes(n):
+    w = W.make("C2", n_queries=4096)
+    w.task, w.slo_us, w.min_acc_bp = w.task[:n], w.slo_us[:n], w.min_acc_bp[:n]
+    if n == 0:
+        import paper_1905_13348_b200 as P
+        cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+        P.infaas_select_batch(cat, None, None, None, None, n=0)
+        P.infaas_load_update(cat, None, 1000, n=0)
+        assert_state_equal(cat, _advance(OracleCatalog(w.rows, w.n_tasks), 1000))
+        cat.free()
+        return
+    run_both(w)
+
+
+def _advance(o, window_us):
+    o.load_update(np.zeros(0, np.uint32), window_us)
+    return o
+
+
+def test_invalid_and_extreme_queries():
+    # tasks 0 and 2 have variants, task 1 has none, tasks >= 3 do not exist
+    rows = rows_from([0, 0, 2, 2, 2], [1, 4, 1, 2, 65535], [100, 2**32 - 1, 50, 1, 7],
+                     [7000, 10000, 0, 6500, 9000], [5, 2**32 - 1, 1, 2, 3], [0, 2**32 - 1, 3, 0, 9])
+    rng = np.random.default_rng(0)
+    n = 5000
+    task = rng.integers(0, 6, n).astype(np.uint16)
+    task[:4] = [65535, 3, 1, 0]
+    slo = rng.choice(np.array([0, 1, 49, 50, 100, 200, 2**32 - 1], np.uint32), n)
+    acc = rng.choice(np.array([0, 6500, 7000, 7001, 10000, 10001, 65535], np.uint16), n)
+    w = W.Workload("edge", 3, rows, task, slo, acc, 0, 0, "edge cases")
+    run_both(w)
+    d = OracleCatalog(rows, 3).select(task, slo, acc)
+    assert (d == INVALID).any() and ((d >> 31) == 1).any() and ((d >> 31) == 0).any()
+
+
+def test_ties_everywhere():
+    # tiny attribute ranges: many equal costs, latencies and accuracies -> tie-break order
+    rng = np.random.default_rng(5)
+    nv, T = 600, 3
+    rows = rows_from(rng.integers(0, T, nv), rng.choice([1, 2], nv), rng.integers(10, 14, nv),
+                     rng.integers(7000, 7004, nv), rng.integers(1, 4, nv), rng.integers(0, 3, nv))
+    n = 30000
+    w = W.Workload("ties", T, rows, rng.integers(0, T, n).astype(np.uint16),
+                   rng.integers(8, 45, n).astype(np.uint32),
+                   rng.integers(6998, 7006, n).astype(np.uint16), 6000, 20, "ties")
+    run_both(w)
+
+
+def test_single_task_maximum_size_and_unequal_tasks():
+    rng = np.random.default_rng(6)
+    sizes = [8192, 1, 0, 37]                        # the per-task limit, a singleton, an empty task
+    task = np.repeat(np.arange(4), sizes)
+    nv = task.size
+    rows = rows_from(task, rng.choice([1, 8, 64], nv), rng.integers(100, 10**6, nv),
+                     rng.integers(5000, 9000, nv), rng.integers(1, 5000, nv))
+    rows = rows[rng.permutation(nv)]
+    n = 20000
+    w = W.Workload("big-task", 4, rows, rng.integers(0, 4, n).astype(np.uint16),
+                   rng.integers(50, 2 * 10**6, n).astype(np.uint32),
+                   rng.integers(5000, 9200, n).astype(np.uint16), 0, 0, "one task at the size limit")
+    run_both(w, check_state=True)
+
+
+def test_load_update_ignores_flagged_and_out_of_range_decisions():
+    import paper_1905_13348_b200 as P
+    w = W.make("C2", n_queries=16)
+    rng = np.random.default_rng(9)
+    dec = rng.integers(0, w.n_variants, 40001).astype(np.uint32)
+    dec[::7] |= NO_FEASIBLE_BIT
+    dec[::11] = INVALID
+    dec[::13] = w.n_variants + 5                     # not a variant id: counted as invalid
+    dec[5:3000] = 17                                  # one hot variant
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    for _ in range(3):
+        P.infaas_load_update(cat, _to_dev(dec), 5000)
+        o.load_update(dec, 5000)
+        assert_state_equal(cat, o)
+    cat.free()
+
+
+def test_frontier_lists_are_sorted_non_dominated_sets():
+    import paper_1905_13348_b200 as P
+    w = W.make("C3", n_queries=16)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    pred = o.pred_lat().astype(np.int64)
+    acc, cost = w.rows["acc_bp"].astype(np.int64), w.rows["cost"].astype(np.int64)
+    for t in range(0, w.n_tasks, 9):
+        ids = P.infaas_catalog_get_frontier(cat, t).astype(np.int64)
+        members = np.flatnonzero(w.rows["task"] == t)
+        keys = [(cost[v], pred[v], -acc[v], v) for v in ids]
+        assert keys == sorted(keys) and set(ids) <= set(members)
+        def dominated(b):
+            return any(pred[a] <= pred[b] and acc[a] >= acc[b] and cost[a] <= cost[b] and
+                       ((pred[a], acc[a], cost[a]) != (pred[b], acc[b], cost[b]) or a < b)
+                       for a in members if a != b)
+        assert set(ids) == {int(v) for v in members if not dominated(v)}
+    cat.free()
+
+
+def test_alignment_and_null_errors():
+    import paper_1905_13348_b200 as P
+    from paper_1905_13348_b200 import binding as B
+    torch = _torch()
+    w = W.make("C1")
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    d_task, d_slo, d_acc = _to_dev(w.task), _to_dev(w.slo_us), _to_dev(w.min_acc_bp)
+    d_dec = torch.zeros(w.n_queries, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.InfaasError) as e:
+        P.infaas_select_batch(cat, d_task[1:], d_slo[1:], d_acc[1:], d_dec[1:])
+    assert e.value.code == -8
+    with pytest.raises(B.InfaasError) as e:
+        P.infaas_select_batch(cat, d_task, None, d_acc, d_dec, n=8)
+    assert e.value.code == -1
+    cat.free()
