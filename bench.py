@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the batched model-variant selection path.
+
+One step = one pass of the whole path over the 16M-query configuration (C3): one
+`infaas_select_batch` over all 2^24 queries against the current load snapshot, then one
+`infaas_load_update` that tallies those decisions, advances every queue by the time the
+batch spans (256 windows' worth) and rebuilds the scan lists.  `value` is queries decided
+per second with inputs resident in HBM; `e2e` repeats it with host buffers and the copies
+inside the timed region.  The per-window pipeline (one update every 65,536 queries) and
+the selection kernel alone are reported beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "queries decided/sec"
+UNIT = "queries/s"
+ALGO_BYTES_PER_QUERY = 12          # 2 (task) + 4 (slo) + 2 (min acc) read, 4 (decision) written
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one selection-kernel launch, from the ncu
+# capture summarised under profiles/ (bytes per query x queries of a launch); None until a
+# capture of the current kernel exists.
+NCU_TRAFFIC_BYTES_PER_QUERY = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3", choices=["C2", "C3", "C4", "C5"])
+    ap.add_argument("--queries", type=int, default=0, help="override the query count (testing)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the windowed / e2e legs")
+    return ap.parse_args()
+
+
+def make_workload(name: str, queries: int):
+    from paper_1905_13348_b200 import workloads as W
+    if name == "C5":
+        kw = {"n_windows": max(1, queries // 65536)} if queries else {}
+    else:
+        kw = {"n_queries": queries} if queries else {}
+    return W.make(name, **kw)
+
+
+def batch_window_us(w) -> int:
+    """Length of the time the whole query array spans (all its windows)."""
+    if w.window:
+        return min(2**32 - 1, max(1, w.n_queries // w.window) * w.window_us)
+    return 1_000_000
+
+
+def workload_config(w) -> dict:
+    return {"workload": f"{w.name}: {w.recipe}", "n_tasks": w.n_tasks, "n_variants": w.n_variants,
+            "n_queries": w.n_queries, "window_queries": w.window, "window_us": w.window_us}
+
+
+# ----------------------------------------------------------------------------------------
+# clocks (read-only sampling during the timed region)
+# ----------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap", 0x80: "hw_power_brake", 0x2: "applications_clocks_setting"}
+
+    def __init__(self, cuda_index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(cuda_index).uuid)
+            uuid = uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM)
+        except Exception as e:  # sampling is best effort
+            self.error = repr(e)
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                bits = nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)
+                for b, name in self.REASONS.items():
+                    if bits & b:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._h is not None:
+            self._t.join()
+
+    def summary(self) -> dict:
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def measured_hbm_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------
+# CPU oracle legs (the only place the benchmark touches oracle/)
+# ----------------------------------------------------------------------------------------
+def oracle_step(o, w, lo, hi, threads, window_us):
+    d = o.select(w.task[lo:hi], w.slo_us[lo:hi], w.min_acc_bp[lo:hi], threads)
+    o.load_update(d, window_us)
+    return d
+
+
+def cpu_baseline(w, target_s: float = 12.0) -> dict:
+    """The oracle as it stands, on this host's cores, on a prefix of the same workload."""
+    from oracle import OracleCatalog
+    threads = os.cpu_count() or 1
+    o = OracleCatalog(w.rows, w.n_tasks)
+    probe = min(w.n_queries, 1 << 18)
+    t0 = time.perf_counter()
+    oracle_step(o, w, 0, probe, threads, 1000)
+    rate = probe / max(1e-9, time.perf_counter() - t0)
+    n = int(min(w.n_queries, max(probe, rate * target_s)))
+    o = OracleCatalog(w.rows, w.n_tasks)
+    t0 = time.perf_counter()
+    oracle_step(o, w, 0, n, threads, batch_window_us(w))
+    dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": f"first {n} of {w.n_queries} queries of {w.name}, select + load update, "
+                      f"{dt:.1f} s"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import OracleCatalog
+    w = make_workload(args.workload, args.queries)
+    threads = os.cpu_count() or 1
+    o = OracleCatalog(w.rows, w.n_tasks)
+    probe = min(w.n_queries, 1 << 18)
+    t0 = time.perf_counter()
+    oracle_step(o, w, 0, probe, threads, 1000)
+    rate = probe / max(1e-9, time.perf_counter() - t0)
+    total_steps = args.steps + args.warmup
+    per_step = int(min(w.n_queries, max(1 << 14, rate * 90.0 / max(1, total_steps))))
+    o = OracleCatalog(w.rows, w.n_tasks)
+    wus = max(1, int(batch_window_us(w) * per_step / w.n_queries))
+    for _ in range(args.warmup):
+        oracle_step(o, w, 0, per_step, threads, wus)
+    t0 = time.perf_counter()
+    for k in range(args.steps):
+        lo = (k * per_step) % max(1, w.n_queries - per_step + 1)
+        oracle_step(o, w, lo, lo + per_step, threads, wus)
+    dt = time.perf_counter() - t0
+    value = args.steps * per_step / dt
+    sample = f"{per_step} queries of {w.name} per step (select + load update)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u32",
+        "data": "synthetic", "config": workload_config(w),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+# ----------------------------------------------------------------------------------------
+# the CUDA path
+# ----------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_1905_13348_b200 as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = make_workload(args.workload, args.queries)
+    n = w.n_queries
+    wus_batch = batch_window_us(w)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks, local)
+
+    def dev_i(a, view):
+        return torch.from_numpy(a.view(view)).to(dev)
+
+    # two rotating copies of the inputs: the working set (2 x 8 B + 4 B per query) is far
+    # larger than L2, so no step starts with its inputs cached
+    inputs = [(dev_i(w.task, np.int16), dev_i(w.slo_us, np.int32), dev_i(w.min_acc_bp, np.int16))
+              for _ in range(2)]
+    d_dec = torch.empty(n, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(k, evs=None):
+        t, s, a = inputs[k & 1]
+        if evs is not None:
+            evs[0].record(stream)
+        P.infaas_select_batch(cat, t, s, a, d_dec, stream=stream)
+        if evs is not None:
+            evs[1].record(stream)
+        P.infaas_load_update(cat, d_dec, wus_batch, stream=stream)
+        if evs is not None:
+            evs[2].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for k in range(max(3, args.warmup)):
+        step(k)
+    P.infaas_catalog_get_state(cat)          # also resizes the staging buffer to the live lists
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    with ClockSampler(local) as clocks:
+        for k in range(args.steps):
+            step(k, evs[k])
+        barrier()
+    total_ms = evs[0][0].elapsed_time(evs[-1][2])
+    sel_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    upd_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    if world > 1:
+        tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    ms_per_step = total_ms / args.steps
+    value = world * n / (ms_per_step * 1e-3)
+    state = P.infaas_catalog_get_state(cat)
+    dec_host = d_dec.cpu().numpy().view(np.uint32)
+
+    peak, peak_kind = measured_hbm_peak()
+    sel_avg_ms = sum(sel_ms) / len(sel_ms)
+    achieved = ALGO_BYTES_PER_QUERY * n / (sel_avg_ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": dict(workload_config(w), step="select_batch(all queries) + load_update(all decisions)",
+                       l2="two rotating input sets; per-step working set 12 B/query > 126 MB L2, no flush",
+                       parallelism="replicas only" if world > 1 else "1 gpu"),
+        "gpu_launches": 3 * args.steps,
+        "kernels_ms": {"select": sel_avg_ms, "select_median": statistics.median(sel_ms),
+                       "tally_plus_rebuild": sum(upd_ms) / len(upd_ms)},
+        "roofline": {"bound": "hbm", "kernel": "select_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": None if NCU_TRAFFIC_BYTES_PER_QUERY is None
+                     else NCU_TRAFFIC_BYTES_PER_QUERY * n},
+        "clocks": clocks.summary(),
+        "decisions": {"feasible": int(((dec_host >> 31) == 0).sum()),
+                      "no_feasible": int((((dec_host >> 31) == 1) & (dec_host != 0xFFFFFFFF)).sum()),
+                      "invalid": int((dec_host == 0xFFFFFFFF).sum()),
+                      "queued_max": int(state["queued"].max())},
+    }
+
+    if not args.no_extras:
+        out["select_only"] = {"value": world * n / (sel_avg_ms * 1e-3), "unit": UNIT, "ms": sel_avg_ms}
+        out["e2e"] = e2e_leg(P, cat, w, dev, wus_batch, max(3, min(10, args.steps)), world, dist)
+        if w.window:
+            out["windowed"] = windowed_leg(P, cat, w, inputs[0], d_dec, world)
+    else:
+        out["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(w)
+    cat.free()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+def e2e_leg(P, cat, w, dev, wus_batch, steps, world, dist):
+    """Same step with HOST inputs and outputs: pinned host arrays are copied to the device,
+    decided, and the decisions copied back, all inside the timed region.  The copies are
+    chunked over two streams so that upload, kernels and download overlap."""
+    import torch
+    n = w.n_queries
+    h_task = torch.from_numpy(w.task.view(np.int16)).pin_memory()
+    h_slo = torch.from_numpy(w.slo_us.view(np.int32)).pin_memory()
+    h_acc = torch.from_numpy(w.min_acc_bp.view(np.int16)).pin_memory()
+    h_dec = torch.empty(n, dtype=torch.int32).pin_memory()
+    d_task = torch.empty(n, dtype=torch.int16, device=dev)
+    d_slo = torch.empty(n, dtype=torch.int32, device=dev)
+    d_acc = torch.empty(n, dtype=torch.int16, device=dev)
+    d_dec = torch.empty(n, dtype=torch.int32, device=dev)
+    chunk = 1 << 21
+    streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    main = torch.cuda.current_stream()
+
+    def step():
+        for s in streams:
+            s.wait_stream(main)
+        for i, lo in enumerate(range(0, n, chunk)):
+            hi = min(n, lo + chunk)
+            s = streams[i & 1]
+            with torch.cuda.stream(s):
+                d_task[lo:hi].copy_(h_task[lo:hi], non_blocking=True)
+                d_slo[lo:hi].copy_(h_slo[lo:hi], non_blocking=True)
+                d_acc[lo:hi].copy_(h_acc[lo:hi], non_blocking=True)
+                P.infaas_select_batch(cat, d_task[lo:hi], d_slo[lo:hi], d_acc[lo:hi], d_dec[lo:hi], stream=s)
+                h_dec[lo:hi].copy_(d_dec[lo:hi], non_blocking=True)
+        for s in streams:
+            main.wait_stream(s)
+        P.infaas_load_update(cat, d_dec, wus_batch, stream=main)
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([dt], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t.item())
+    return {"value": world * n * steps / dt, "unit": UNIT, "h2d_bytes_per_step": 8 * n,
+            "d2h_bytes_per_step": 4 * n, "ms_per_step": 1e3 * dt / steps, "steps": steps,
+            "how": "pinned host -> device copies, select per 2M-query chunk on two streams, "
+                   "decisions copied back, one load update; host wall clock around synchronize"}
+
+
+def windowed_leg(P, cat, w, inp, d_dec, world):
+    """The workload as a stream of windows: select one window, update the load, repeat."""
+    import torch
+    t, s, a = inp
+    W_ = w.window
+    nwin = w.n_queries // W_
+    stream = torch.cuda.current_stream()
+
+    def run():
+        for k in range(nwin):
+            lo, hi = k * W_, (k + 1) * W_
+            P.infaas_select_batch(cat, t[lo:hi], s[lo:hi], a[lo:hi], d_dec[lo:hi], stream=stream)
+            P.infaas_load_update(cat, d_dec[lo:hi], w.window_us, stream=stream)
+
+    run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 3
+    e0.record(stream)
+    for _ in range(reps):
+        run()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    return {"value": world * nwin * W_ / (ms * 1e-3), "unit": UNIT, "windows": nwin,
+            "window_queries": W_, "us_per_window": 1e3 * ms / nwin, "gpu_launches_per_window": 3}
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
