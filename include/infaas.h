@@ -134,6 +134,31 @@ int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_
 int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_ids,
                                 uint32_t cap, uint32_t *h_len, void *cuda_stream);
 
+/* (No counterpart in the paper: an addition for callers that cannot allocate.)
+ * Per-variant tallies of a decision array, as the first step of infaas_load_update computes
+ * them, for callers that must not trigger a device allocation: a serving process that has
+ * handed all free device memory to its own pool (a cudaMalloc there fails), or a dispatch
+ * loop that cannot afford the device-wide stall an allocation causes.  It needs no catalog
+ * handle and calls no cudaMalloc / cudaFree nor any allocating routine: its scratch (the
+ * counters it accumulates into) is a fixed array inside the library's device image, which
+ * every GPU that loads the library holds until the process exits (256 KB + 32 B).
+ *     d_count[v]    = #{q : d_decision[q] == v}      for v < n_variants (bit 31 clear)
+ *     d_counters[3] = decisions tallied, decisions with bit 31 set (not INFAAS_INVALID),
+ *                     invalid decisions (INFAAS_INVALID or an id >= n_variants)
+ *   d_decision   DEVICE, n u32, 16-byte aligned, read only; n <= 2^32-1.
+ *   n_variants   1 .. INFAAS_STATIC_MAX_VARIANTS, else INFAAS_E_TOO_LARGE.
+ *   d_count      DEVICE, n_variants u32, overwritten.   d_counters  DEVICE, 3 u64, overwritten.
+ *   cuda_device  device the arrays live on (0..63).      cuda_stream a cudaStream_t on it.
+ * Asynchronous and stream-ordered.  The first call on each device looks up the array's
+ * device address (a set-up step): make that first call outside any stream capture.  All
+ * calls on a device share the one array and each call clears what it uses before counting,
+ * so two calls whose work overlaps on the GPU (different streams, no ordering) race and give
+ * wrong counts; order them.  Errors: E_NULL, E_ALIGN, E_TOO_LARGE, E_CUDA. */
+#define INFAAS_STATIC_MAX_VARIANTS 65536u
+int infaas_tally_static(const uint32_t *d_decision, uint64_t n, uint32_t n_variants,
+                        uint32_t *d_count, uint64_t *d_counters, int cuda_device,
+                        void *cuda_stream);
+
 /* Release the catalog and its device memory.  NULL is allowed. */
 void infaas_catalog_free(infaas_catalog *c);
 

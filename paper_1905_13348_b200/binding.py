@@ -21,7 +21,7 @@ _lib = None
 
 EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
-           "infaas_strerror", "infaas_last_cuda_error")
+           "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static")
 
 
 class InfaasError(RuntimeError):
@@ -52,6 +52,8 @@ def _load():
     for name in ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
                  "infaas_catalog_get_state", "infaas_catalog_get_frontier"):
         getattr(lib, name).restype = i32
+    lib.infaas_tally_static.argtypes = [vp, u64, u32, vp, vp, i32, vp]
+    lib.infaas_tally_static.restype = i32
     lib.infaas_strerror.argtypes = [i32]
     lib.infaas_strerror.restype = ctypes.c_char_p
     lib.infaas_last_cuda_error.argtypes = []
@@ -145,3 +147,18 @@ def infaas_catalog_get_frontier(cat: Catalog, task: int, stream=None) -> np.ndar
                                                ctypes.byref(ln), _stream_ptr(stream)),
            "infaas_catalog_get_frontier")
     return ids[:ln.value].copy()
+
+
+def infaas_tally_static(d_decision, n_variants: int, d_count, d_counters, n=None, stream=None) -> None:
+    """Allocation-free tallies: d_count (int32/uint32 CUDA tensor of n_variants) and
+    d_counters (int64 CUDA tensor of 3) are overwritten; see include/infaas.h."""
+    import torch
+    n = int(d_decision.shape[0]) if n is None else int(n)
+    if not (d_counters.is_cuda and d_counters.is_contiguous() and d_counters.dtype in (torch.int64, torch.uint64)
+            and d_counters.numel() >= 3):
+        raise TypeError("d_counters must be a contiguous CUDA tensor of 3 64-bit integers")
+    if d_count.numel() < n_variants:
+        raise ValueError("d_count is shorter than n_variants")
+    _check(_load().infaas_tally_static(_dev_ptr(d_decision, "u32"), n, int(n_variants),
+                                       _dev_ptr(d_count, "u32"), d_counters.data_ptr(),
+                                       d_count.device.index, _stream_ptr(stream)), "infaas_tally_static")
