@@ -362,31 +362,45 @@ def e2e_leg(P, cat, w, dev, wus_batch, steps, world, dist):
 
 
 def windowed_leg(P, cat, w, inp, d_dec, world):
-    """The workload as a stream of windows: select one window, update the load, repeat."""
+    """The workload as a stream of windows: select one window, update the load, repeat.
+    All windows are captured once into a CUDA graph (the calls only launch kernels), so the
+    timing shows the device-side dependency chain and not the Python call overhead."""
     import torch
     t, s, a = inp
     W_ = w.window
     nwin = w.n_queries // W_
-    stream = torch.cuda.current_stream()
+    side = torch.cuda.Stream()
 
-    def run():
+    def run(stream):
         for k in range(nwin):
             lo, hi = k * W_, (k + 1) * W_
             P.infaas_select_batch(cat, t[lo:hi], s[lo:hi], a[lo:hi], d_dec[lo:hi], stream=stream)
             P.infaas_load_update(cat, d_dec[lo:hi], w.window_us, stream=stream)
 
-    run()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = 3
-    e0.record(stream)
-    for _ in range(reps):
-        run()
-    e1.record(stream)
-    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        run(side)                      # plain pass first (also warms the kernels up)
+        side.synchronize()
+        t0 = time.perf_counter()
+        run(side)
+        side.synchronize()
+        eager_ms = 1e3 * (time.perf_counter() - t0)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            run(side)
+        graph.replay()
+        side.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 5
+        e0.record(side)
+        for _ in range(reps):
+            graph.replay()
+        e1.record(side)
+        side.synchronize()
     ms = e0.elapsed_time(e1) / reps
     return {"value": world * nwin * W_ / (ms * 1e-3), "unit": UNIT, "windows": nwin,
-            "window_queries": W_, "us_per_window": 1e3 * ms / nwin, "gpu_launches_per_window": 3}
+            "window_queries": W_, "us_per_window": 1e3 * ms / nwin, "gpu_launches_per_window": 3,
+            "how": "CUDA graph of all windows", "us_per_window_python_calls": 1e3 * eager_ms / nwin}
 
 
 def main():

@@ -16,8 +16,8 @@ struct infaas_catalog {
   void *arena = nullptr;                 // one device allocation holds every array
   std::vector<uint32_t> slot_of_id;      // host copy, for get_state
   std::vector<uint32_t> task_off, reg_off;
-  uint32_t select_smem = 0;              // dynamic shared memory given to the selection kernel
-  uint32_t worst_blob_bytes = 0;         // image size if no variant were dominated
+  uint32_t select_smem = 0;              // shared memory reserved for the staged image
+  uint32_t worst_image_bytes = 0;        // image size if every block had its largest size
 };
 
 namespace {
@@ -61,12 +61,12 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // with headroom for growth between two such refreshes.
 int refresh_select_plan(infaas_catalog *c, cudaStream_t stream) {
   uint32_t hdr[4] = {0, 0, 0, 0};
-  CUDA_TRY(cudaMemcpyAsync(hdr, c->d.blob_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, stream));
+  CUDA_TRY(cudaMemcpyAsync(hdr, c->d.image_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, stream));
   CUDA_TRY(cudaStreamSynchronize(stream));
   uint64_t want = (uint64_t)hdr[0] + hdr[0] / 2 + 4096;
-  if (want > c->worst_blob_bytes) want = c->worst_blob_bytes;
-  if (want > infaas::SELECT_MAX_SMEM) want = infaas::SELECT_MAX_SMEM;
-  c->select_smem = (uint32_t)(want & ~(uint64_t)15);
+  if (want > c->worst_image_bytes) want = c->worst_image_bytes;
+  if (want > infaas::SELECT_MAX_SMEM) want = infaas::SELECT_MAX_SMEM;   // the launcher trims further
+  c->select_smem = (uint32_t)((want + 15) & ~(uint64_t)15);
   return INFAAS_OK;
 }
 
@@ -116,9 +116,12 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   }
   if (max_task > INFAAS_MAX_TASK_VARIANTS) return INFAAS_E_TOO_LARGE;
   std::vector<uint32_t> reg_off(n_tasks + 1, 0);
-  for (uint32_t t = 0; t < n_tasks; ++t)
-    reg_off[t + 1] = reg_off[t] + (uint32_t)round_up(task_off[t + 1] - task_off[t], 4);
-  const uint32_t region_entries = reg_off[n_tasks];
+  uint64_t region_bytes = 0;
+  for (uint32_t t = 0; t < n_tasks; ++t) {
+    region_bytes += infaas::block_capacity(task_off[t + 1] - task_off[t]);
+    if (region_bytes > 0xF0000000ull) return INFAAS_E_TOO_LARGE;
+    reg_off[t + 1] = (uint32_t)region_bytes;
+  }
 
   std::vector<uint32_t> h_lat(n_variants), h_cost(n_variants), h_id(n_variants), h_queued(n_variants),
       slot_of_id(n_variants);
@@ -140,9 +143,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   if (scope.status != cudaSuccess) { delete c; return cuda_fail(scope.status); }
 
   // ---- one arena, carved into 256-byte aligned arrays ----
-  const uint32_t n_tasks_pad = (n_tasks + 1u) & ~1u;
-  const uint64_t worst_blob = (uint64_t)n_tasks_pad * 8u + (uint64_t)round_up(n_variants, 4) * 12u;
-  if (worst_blob > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
+  const uint64_t worst_image = (uint64_t)n_tasks * sizeof(infaas::TaskDesc) + region_bytes;
+  if (worst_image > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
   size_t total = 0;
   auto carve = [&total](size_t bytes) { size_t off = total; total += round_up(bytes, 256); return off; };
   const size_t o_task_off = carve((n_tasks + 1) * 4), o_reg_off = carve((n_tasks + 1) * 4);
@@ -151,9 +153,9 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_id = carve((size_t)n_variants * 4), o_queued = carve((size_t)n_variants * 4);
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
-  const size_t o_fkey = carve((size_t)region_entries * 8), o_fid = carve((size_t)region_entries * 4);
-  const size_t o_flen = carve((size_t)n_tasks * 4);
-  const size_t o_blob = carve((size_t)worst_blob), o_hdr = carve(16);
+  const size_t o_regions = carve((size_t)region_bytes);
+  const size_t o_flen = carve((size_t)n_tasks * 4), o_fmeta = carve((size_t)n_tasks * 4);
+  const size_t o_image = carve((size_t)worst_image), o_hdr = carve(16);
   const size_t o_counters = carve(24), o_done = carve(4), o_err = carve(4);
 
 #define LOAD_TRY(expr)                                                     \
@@ -180,9 +182,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   DeviceCatalog &d = c->d;
   d.n_variants = n_variants;
   d.n_tasks = n_tasks;
-  d.n_tasks_pad = n_tasks_pad;
   d.max_task_variants = max_task;
-  d.region_entries = region_entries;
   d.task_off = reinterpret_cast<const uint32_t *>(base + o_task_off);
   d.reg_off = reinterpret_cast<const uint32_t *>(base + o_reg_off);
   d.s_lat = reinterpret_cast<const uint32_t *>(base + o_lat);
@@ -194,19 +194,19 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.s_pred = reinterpret_cast<uint32_t *>(base + o_pred);
   d.s_served = reinterpret_cast<unsigned long long *>(base + o_served);
   d.count_by_id = reinterpret_cast<uint32_t *>(base + o_count);
-  d.f_key = reinterpret_cast<unsigned long long *>(base + o_fkey);
-  d.f_id = reinterpret_cast<uint32_t *>(base + o_fid);
+  d.regions = base + o_regions;
   d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
-  d.blob = base + o_blob;
-  d.blob_capacity = (uint32_t)worst_blob;
-  d.blob_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
+  d.f_meta = reinterpret_cast<uint32_t *>(base + o_fmeta);
+  d.image = base + o_image;
+  d.image_capacity = (uint32_t)worst_image;
+  d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
   d.counters = reinterpret_cast<unsigned long long *>(base + o_counters);
   d.done_ctr = reinterpret_cast<uint32_t *>(base + o_done);
   d.err = reinterpret_cast<uint32_t *>(base + o_err);
   c->slot_of_id.swap(slot_of_id);
   c->task_off.swap(task_off);
   c->reg_off.swap(reg_off);
-  c->worst_blob_bytes = (uint32_t)worst_blob;
+  c->worst_image_bytes = (uint32_t)worst_image;
 
   LOAD_TRY(infaas::prepare_select_kernel());
   LOAD_TRY(infaas::prepare_rebuild_kernel());
@@ -307,8 +307,8 @@ int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_id
   *h_len = len;
   const uint32_t ncopy = len < cap ? len : cap;
   if (h_ids && ncopy) {
-    CUDA_TRY(cudaMemcpyAsync(h_ids, c->d.f_id + c->reg_off[task], (size_t)ncopy * 4,
-                             cudaMemcpyDeviceToHost, s));
+    const unsigned char *ids = c->d.regions + c->reg_off[task] + infaas::block_layout(len).ids;
+    CUDA_TRY(cudaMemcpyAsync(h_ids, ids, (size_t)ncopy * 4, cudaMemcpyDeviceToHost, s));
     CUDA_TRY(cudaStreamSynchronize(s));
   }
   return INFAAS_OK;

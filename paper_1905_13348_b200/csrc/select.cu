@@ -3,21 +3,31 @@
 // (Section 4.1 of the paper, "Case I: on arrival of a query"; cost objective as in the
 // worked example of Section 2.2).
 //
-// The per-task scan lists are already sorted by (cost, pred_lat, -acc, id) and pruned to
-// non-dominated variants, so the answer for a feasible query is the FIRST list entry that
-// meets both requirements, and the nearest miss is the first entry with the smallest
-// distance.  All lists together are a few tens of KB: each CTA stages the packed image in
-// shared memory with bulk asynchronous copies (TMA, mbarrier completion) once and then
-// streams queries through it, four per thread per iteration with 128-bit loads and stores.
+// Each task's scan list is sorted by (cost, pred_lat, -acc, id) and pruned to non-dominated
+// variants, so the answer for a feasible query is the FIRST list position that meets both
+// requirements.  Instead of walking the list, a thread ranks the query's SLO among the
+// list's latencies and its minimum accuracy among the list's accuracies (bucket table +
+// a short refine loop) and ANDs two precomputed position bitmasks; the lowest set bit is
+// the answer (layout in common.cuh).  The packed image of all tasks is staged in shared
+// memory once per CTA with bulk asynchronous copies (TMA, mbarrier completion); queries
+// stream through with 128-bit loads and stores, four per thread and iteration.
+// Queries without a feasible variant (a few percent) are parked in a per-warp list and
+// resolved 32 at a time with all lanes busy: a pass over the list computing the distance
+// d = 10^4 * over_lat + slo * under_acc.
 #include "common.cuh"
 
 namespace infaas {
 
 namespace {
 
-constexpr int SELECT_THREADS = 512;
+constexpr int SELECT_THREADS = 1024;
+constexpr int SELECT_WARPS = SELECT_THREADS / 32;
+constexpr uint32_t WARP_TILE = 128;              // queries per warp and iteration
+constexpr uint32_t PARK_CAP = 32 + WARP_TILE;    // parked queries per warp
+constexpr uint32_t PARK_BYTES = SELECT_WARPS * PARK_CAP * 4;
 constexpr uint32_t STAGE_CHUNK = 32768;          // bytes per bulk copy
 constexpr uint32_t STAGE_POLL_LIMIT = 1u << 22;  // bounded wait on the staging barrier
+constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-3)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -25,8 +35,8 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p) {
 
 // Stage `bytes` (multiple of 16) from global `src` (16-byte aligned) into shared `dst`.
 // Returns false if the copy did not complete within the poll limit.
-__device__ __forceinline__ bool stage_blob(unsigned char *dst, const unsigned char *src,
-                                           uint32_t bytes, unsigned long long *mbar) {
+__device__ __forceinline__ bool stage_image(unsigned char *dst, const unsigned char *src,
+                                            uint32_t bytes, unsigned long long *mbar) {
   const uint32_t bar = smem_u32(mbar);
   if (threadIdx.x == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
@@ -57,88 +67,230 @@ __device__ __forceinline__ bool stage_blob(unsigned char *dst, const unsigned ch
   return __syncthreads_and((int)done) != 0;
 }
 
-// One query against its task's list.  table/keys/ids point to shared memory (staged) or to
-// the global image.
-__device__ __forceinline__ uint32_t decide(const uint2 *__restrict__ table,
-                                           const unsigned long long *__restrict__ keys,
-                                           const uint32_t *__restrict__ ids, uint32_t n_tasks,
-                                           uint32_t task, uint32_t slo, uint32_t min_acc) {
-  if (task >= n_tasks) return INFAAS_INVALID;
-  const uint2 sl = table[task];
-  const uint32_t start = sl.x, len = sl.y;
-  if (len == 0) return INFAAS_INVALID;
-  const unsigned long long *k = keys + start;
-  for (uint32_t i = 0; i < len; ++i) {
-    const unsigned long long e = k[i];
-    if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return ids[start + i];
+// The image, read either from shared memory (32-bit addresses, ld.shared) or from global
+// memory (read-only path).  Offsets are bytes from the start of the image.
+struct SharedImage {
+  uint32_t base;
+  __device__ __forceinline__ uint32_t u8(uint32_t off) const {
+    uint32_t v; asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
   }
-  // nothing meets both: nearest miss, d = 10^4 * over_lat + slo * under_acc (64-bit);
-  // strict '<' keeps the first of equal distances, i.e. the smallest (cost, pred, -acc, id)
+  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
+    uint32_t v; asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
+  }
+  __device__ __forceinline__ uint32_t u32(uint32_t off) const {
+    uint32_t v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
+  }
+  __device__ __forceinline__ unsigned long long u64(uint32_t off) const {
+    unsigned long long v; asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(base + off)); return v;
+  }
+  __device__ __forceinline__ uint4 v4(uint32_t off) const {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(base + off));
+    return v;
+  }
+};
+
+struct GlobalImage {
+  const unsigned char *base;
+  __device__ __forceinline__ uint32_t u8(uint32_t off) const { return __ldg(base + off); }
+  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
+    return __ldg(reinterpret_cast<const uint16_t *>(base + off));
+  }
+  __device__ __forceinline__ uint32_t u32(uint32_t off) const {
+    return __ldg(reinterpret_cast<const uint32_t *>(base + off));
+  }
+  __device__ __forceinline__ unsigned long long u64(uint32_t off) const {
+    return __ldg(reinterpret_cast<const unsigned long long *>(base + off));
+  }
+  __device__ __forceinline__ uint4 v4(uint32_t off) const {
+    return __ldg(reinterpret_cast<const uint4 *>(base + off));
+  }
+};
+
+// First list position that meets (slo, min_acc), as a decision; PENDING if none does.
+template <class Img>
+__device__ __forceinline__ uint32_t decide(const Img &img, uint32_t n_tasks, uint32_t task,
+                                           uint32_t slo, uint32_t min_acc) {
+  if (task >= n_tasks) return INFAAS_INVALID;
+  const uint4 d0 = img.v4(task * 32u);        // off_masks, f_nw, acc_meta, off_keys
+  const uint4 d1 = img.v4(task * 32u + 16u);  // off_thr, off_ids, off_accs, off_start
+  const uint32_t F = d0.y & 0xFFFFu, nw = d0.y >> 16;
+  if (F == 0) return INFAAS_INVALID;
+  if (nw == 0) {   // list too long for the index: walk it
+    for (uint32_t i = 0; i < F; ++i) {
+      const unsigned long long e = img.u64(d0.w + 8u * i);
+      if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return img.u32(d1.y + 4u * i);
+    }
+    return PENDING;
+  }
+  // r = #{list latencies <= slo}
+  const uint32_t fb = __float_as_uint(__uint2float_rz(slo)) >> 20;
+  uint32_t r = img.u8(d1.w + max(fb, SLO_BUCKET_BIAS) - SLO_BUCKET_BIAS);
+  while (r < F && img.u32(d1.x + 4u * r) <= slo) ++r;
+  // k = #{list accuracies < min_acc}
+  const uint32_t acc_base = d0.z & 0xFFFFu, acc_shift = d0.z >> 16;
+  const uint32_t above = min_acc > acc_base ? min_acc - acc_base : 0u;
+  uint32_t k = img.u8(d1.w + SLO_BUCKET_BYTES + min(above >> acc_shift, ACC_BUCKETS - 1u));
+  while (k < F && img.u16(d1.z + 2u * k) < min_acc) ++k;
+  // positions that meet both = ML[r] & MA[k]
+  const uint32_t ml = d0.x + 8u * r * nw, ma = d0.x + 8u * ((F + 1u) * nw + k * nw);
+  for (uint32_t w = 0; w < nw; ++w) {
+    const unsigned long long x = img.u64(ml + 8u * w) & img.u64(ma + 8u * w);
+    if (x) return img.u32(d1.y + 4u * (64u * w + (uint32_t)__ffsll((long long)x) - 1u));
+  }
+  return PENDING;
+}
+
+// Nearest miss of a query no list entry meets: d = 10^4 * over_lat + slo * under_acc
+// (64-bit); strict '<' keeps the first of equal distances, i.e. the smallest
+// (cost, pred_lat, -acc, id).
+template <class Img>
+__device__ __forceinline__ uint32_t nearest_miss(const Img &img, uint32_t task, uint32_t slo,
+                                                 uint32_t min_acc) {
+  const uint4 d0 = img.v4(task * 32u);
+  const uint32_t F = d0.y & 0xFFFFu, off_ids = img.u32(task * 32u + 20u);
   unsigned long long best = ~0ull;
   uint32_t best_i = 0;
-  for (uint32_t i = 0; i < len; ++i) {
-    const unsigned long long e = k[i];
+  for (uint32_t i = 0; i < F; ++i) {
+    const unsigned long long e = img.u64(d0.w + 8u * i);
     const uint32_t pred = (uint32_t)e, acc = (uint32_t)(e >> 32);
     const uint32_t over = pred > slo ? pred - slo : 0u;
     const uint32_t under = min_acc > acc ? min_acc - acc : 0u;
     const unsigned long long d = (unsigned long long)over * 10000ull + (unsigned long long)slo * under;
     if (d < best) { best = d; best_i = i; }
   }
-  return INFAAS_NO_FEASIBLE | ids[start + best_i];
+  return INFAAS_NO_FEASIBLE | img.u32(off_ids + 4u * best_i);
 }
 
-__device__ __forceinline__ void select_body(const unsigned char *image, uint32_t n_tasks,
-                                            uint32_t n_tasks_pad, uint32_t e_pad,
-                                            const uint16_t *__restrict__ task,
-                                            const uint32_t *__restrict__ slo,
-                                            const uint16_t *__restrict__ min_acc, uint64_t n,
-                                            uint32_t *__restrict__ decision) {
-  const uint2 *table = reinterpret_cast<const uint2 *>(image);
-  const unsigned long long *keys =
-      reinterpret_cast<const unsigned long long *>(image + blob_table_bytes(n_tasks_pad));
-  const uint32_t *ids = reinterpret_cast<const uint32_t *>(keys + e_pad);
+struct Queries {
+  const uint16_t *__restrict__ task;
+  const uint32_t *__restrict__ slo;
+  const uint16_t *__restrict__ min_acc;
+  uint32_t *__restrict__ decision;
+};
 
-  const uint64_t n4 = n >> 2;
-  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-  const uint2 *task4 = reinterpret_cast<const uint2 *>(task);
-  const uint4 *slo4 = reinterpret_cast<const uint4 *>(slo);
-  const uint2 *acc4 = reinterpret_cast<const uint2 *>(min_acc);
-  uint4 *dec4 = reinterpret_cast<uint4 *>(decision);
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-    const uint2 t = __ldcs(task4 + i);
-    const uint4 s = __ldcs(slo4 + i);
-    const uint2 a = __ldcs(acc4 + i);
+// Resolve up to 32 parked queries, one per lane.  `rel` is the query's offset from `q0`.
+template <class Img>
+__device__ __forceinline__ void resolve_parked(const Img &img, const Queries &q, uint64_t q0,
+                                               const uint32_t *park, uint32_t first, uint32_t count) {
+  const uint32_t lane = threadIdx.x & 31;
+  if (lane < count) {
+    const uint64_t i = q0 + park[first + lane];
+    q.decision[i] = nearest_miss(img, q.task[i], q.slo[i], q.min_acc[i]);
+  }
+}
+
+// Append the lanes with `pending` to the warp's park list (all lanes call this).
+__device__ __forceinline__ void park_append(uint32_t *park, uint32_t &cnt, bool pending, uint32_t rel) {
+  const unsigned m = __ballot_sync(0xFFFFFFFFu, pending);
+  if (pending) park[cnt + __popc(m & ((1u << (threadIdx.x & 31)) - 1u))] = rel;
+  cnt += __popc(m);
+}
+
+template <class Img>
+__device__ __forceinline__ void select_body(const Img &img, uint32_t n_tasks, const Queries &q,
+                                            uint64_t n, uint64_t per_cta, uint32_t *park_all) {
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t *park = park_all + warp * PARK_CAP;
+  uint32_t parked = 0;
+  const uint64_t q0 = (uint64_t)blockIdx.x * per_cta;
+  const uint64_t q1 = min(n, q0 + per_cta);
+  if (q0 >= q1) return;
+  const uint64_t span = q1 - q0;                       // < 2^32 (checked by the launcher)
+  const uint64_t full_tiles = span / WARP_TILE;
+
+  // full tiles: 4 consecutive queries per lane, 128-bit loads, next tile prefetched
+  uint64_t tile = warp;
+  uint2 t4 = make_uint2(0, 0), a4 = make_uint2(0, 0);
+  uint4 s4 = make_uint4(0, 0, 0, 0);
+  if (tile < full_tiles) {
+    const uint64_t i4 = (q0 + tile * WARP_TILE) / 4 + lane;
+    t4 = __ldcs(reinterpret_cast<const uint2 *>(q.task) + i4);
+    s4 = __ldcs(reinterpret_cast<const uint4 *>(q.slo) + i4);
+    a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
+  }
+  for (; tile < full_tiles; tile += SELECT_WARPS) {
+    const uint2 t = t4, a = a4;
+    const uint4 s = s4;
+    const uint64_t next = tile + SELECT_WARPS;
+    if (next < full_tiles) {
+      const uint64_t i4 = (q0 + next * WARP_TILE) / 4 + lane;
+      t4 = __ldcs(reinterpret_cast<const uint2 *>(q.task) + i4);
+      s4 = __ldcs(reinterpret_cast<const uint4 *>(q.slo) + i4);
+      a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
+    }
     uint4 d;
-    d.x = decide(table, keys, ids, n_tasks, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
-    d.y = decide(table, keys, ids, n_tasks, t.x >> 16, s.y, a.x >> 16);
-    d.z = decide(table, keys, ids, n_tasks, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
-    d.w = decide(table, keys, ids, n_tasks, t.y >> 16, s.w, a.y >> 16);
-    __stcs(dec4 + i, d);
+    d.x = decide(img, n_tasks, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
+    d.y = decide(img, n_tasks, t.x >> 16, s.y, a.x >> 16);
+    d.z = decide(img, n_tasks, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
+    d.w = decide(img, n_tasks, t.y >> 16, s.w, a.y >> 16);
+    const uint32_t rel = (uint32_t)(tile * WARP_TILE) + lane * 4u;
+    uint32_t *out = q.decision + q0 + rel;
+    const bool any_pending = d.x == PENDING || d.y == PENDING || d.z == PENDING || d.w == PENDING;
+    if (!any_pending) {
+      __stcs(reinterpret_cast<uint4 *>(out), d);
+    } else {            // a parked slot is written later by another lane: leave it alone now
+      if (d.x != PENDING) out[0] = d.x;
+      if (d.y != PENDING) out[1] = d.y;
+      if (d.z != PENDING) out[2] = d.z;
+      if (d.w != PENDING) out[3] = d.w;
+    }
+    if (__any_sync(0xFFFFFFFFu, any_pending)) {
+      park_append(park, parked, d.x == PENDING, rel);
+      park_append(park, parked, d.y == PENDING, rel + 1);
+      park_append(park, parked, d.z == PENDING, rel + 2);
+      park_append(park, parked, d.w == PENDING, rel + 3);
+      __syncwarp();
+      while (parked >= 32) {
+        parked -= 32;
+        resolve_parked(img, q, q0, park, parked, 32);
+      }
+      __syncwarp();
+    }
   }
-  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) {   // ragged tail
-    const uint64_t q = (n4 << 2) + threadIdx.x;
-    decision[q] = decide(table, keys, ids, n_tasks, task[q], slo[q], min_acc[q]);
+  // ragged tail of the CTA's range (fewer than WARP_TILE queries): one warp, scalar accesses
+  const uint64_t tail0 = full_tiles * WARP_TILE;
+  if (tail0 < span && warp == (uint32_t)(full_tiles % SELECT_WARPS)) {
+    for (uint32_t j = 0; j < WARP_TILE / 32; ++j) {
+      const uint64_t rel = tail0 + j * 32u + lane;
+      uint32_t d = 0;
+      if (rel < span) {
+        const uint64_t i = q0 + rel;
+        d = decide(img, n_tasks, q.task[i], q.slo[i], q.min_acc[i]);
+        if (d != PENDING) q.decision[i] = d;
+      }
+      park_append(park, parked, rel < span && d == PENDING, (uint32_t)rel);
+    }
+    __syncwarp();
+    while (parked >= 32) {
+      parked -= 32;
+      resolve_parked(img, q, q0, park, parked, 32);
+    }
   }
+  __syncwarp();
+  resolve_parked(img, q, q0, park, 0, parked);
 }
 
-__global__ void __launch_bounds__(SELECT_THREADS)
-select_kernel(const unsigned char *__restrict__ blob, const uint32_t *__restrict__ blob_hdr,
-              uint32_t n_tasks, uint32_t n_tasks_pad, uint32_t smem_bytes,
-              const uint16_t *__restrict__ task, const uint32_t *__restrict__ slo,
-              const uint16_t *__restrict__ min_acc, uint64_t n, uint32_t *__restrict__ decision,
+__global__ void __launch_bounds__(SELECT_THREADS, 1)
+select_kernel(const unsigned char *__restrict__ image, const uint32_t *__restrict__ image_hdr,
+              uint32_t n_tasks, uint32_t image_smem, Queries q, uint64_t n, uint64_t per_cta,
               uint32_t *err) {
-  extern __shared__ __align__(128) unsigned char image[];
+  extern __shared__ __align__(128) unsigned char smem[];   // [park lists][staged image]
   __shared__ __align__(8) unsigned long long mbar;
-  const uint32_t bytes = blob_hdr[0], e_pad = blob_hdr[1];
-  if (bytes <= smem_bytes) {
-    if (!stage_blob(image, blob, bytes, &mbar)) {
+  uint32_t *park = reinterpret_cast<uint32_t *>(smem);
+  unsigned char *staged = smem + PARK_BYTES;
+  const uint32_t bytes = image_hdr[0];
+  if (bytes <= image_smem) {
+    if (!stage_image(staged, image, bytes, &mbar)) {
       if (threadIdx.x == 0) atomicMax(err, (uint32_t)DEV_ERR_STAGE_TIMEOUT);
       return;
     }
-    select_body(image, n_tasks, n_tasks_pad, e_pad, task, slo, min_acc, n, decision);
+    SharedImage img{smem_u32(staged)};
+    select_body(img, n_tasks, q, n, per_cta, park);
   } else {
-    // lists do not fit in shared memory: scan them in global memory (L2-resident)
-    select_body(blob, n_tasks, n_tasks_pad, e_pad, task, slo, min_acc, n, decision);
+    // the image does not fit in shared memory: read it from global memory (L1/L2 resident)
+    GlobalImage img{image};
+    select_body(img, n_tasks, q, n, per_cta, park);
   }
 }
 
@@ -151,20 +303,19 @@ cudaError_t prepare_select_kernel() {
 
 cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const uint32_t *d_slo,
                           const uint16_t *d_min_acc, uint64_t n, uint32_t *d_decision,
-                          int sm_count, uint32_t smem_bytes, cudaStream_t stream) {
+                          int sm_count, uint32_t image_smem, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
-  // resident CTAs per SM for this shared-memory size (227 KB usable per SM, 1 KB reserved per CTA)
-  uint32_t per_sm = (uint32_t)(233472u / (smem_bytes + 1024u + 64u));
-  const uint32_t by_threads = 2048 / SELECT_THREADS;
-  if (per_sm > by_threads) per_sm = by_threads;
-  if (per_sm < 1) per_sm = 1;
-  const uint64_t want = ((n >> 2) + SELECT_THREADS - 1) / SELECT_THREADS;
-  uint64_t grid = (uint64_t)sm_count * per_sm;
-  if (grid > want) grid = want;
-  if (grid < 1) grid = 1;
-  select_kernel<<<(uint32_t)grid, SELECT_THREADS, smem_bytes, stream>>>(
-      c.blob, c.blob_hdr, c.n_tasks, c.n_tasks_pad, smem_bytes, d_task, d_slo, d_min_acc, n,
-      d_decision, c.err);
+  if (image_smem + PARK_BYTES > SELECT_MAX_SMEM) image_smem = (SELECT_MAX_SMEM - PARK_BYTES) & ~15u;
+  // one CTA per SM; every CTA takes one contiguous range, a multiple of the warp tile
+  uint64_t grid = (uint64_t)sm_count;
+  const uint64_t tiles = (n + WARP_TILE - 1) / WARP_TILE;
+  if (grid > tiles) grid = tiles;
+  const uint64_t per_cta = (tiles + grid - 1) / grid * WARP_TILE;
+  if (per_cta > 0xFFFFFFFFull) return cudaErrorInvalidValue;
+  grid = (n + per_cta - 1) / per_cta;
+  Queries q{d_task, d_slo, d_min_acc, d_decision};
+  select_kernel<<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(
+      c.image, c.image_hdr, c.n_tasks, image_smem, q, n, per_cta, c.err);
   return cudaGetLastError();
 }
 

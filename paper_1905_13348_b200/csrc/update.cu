@@ -100,12 +100,87 @@ __device__ __forceinline__ uint32_t block_excl_scan_flag(bool flag, uint32_t *wa
   return before + in_warp;
 }
 
+// Smallest slo that falls in SLO bucket b >= 1 (see common.cuh).
+__device__ __forceinline__ uint32_t slo_bucket_floor(uint32_t b) {
+  const float f = __uint_as_float((b + SLO_BUCKET_BIAS) << 20);
+  return (uint32_t)ceilf(f);     // exact: f < 2^32 and has at most 3 fractional bits
+}
+
+// Builds the rank / bitmask index of a list of F <= MASK_MAX_F entries (see common.cuh).
+// fr_pred / fr_acc: the list in scan order (shared memory).  Writes into the task block.
+__device__ void build_index(unsigned char *block, const BlockLayout &L, uint32_t F,
+                            const uint32_t *fr_pred, const uint16_t *fr_acc, uint16_t *rkL,
+                            uint16_t *rkA, uint32_t *thr_s, uint16_t *acc_s, uint32_t *meta_out) {
+  const uint32_t tid = threadIdx.x, B = blockDim.x;
+  // ranks by counting (stable: equal values keep scan order)
+  for (uint32_t p = tid; p < F; p += B) {
+    const uint32_t pp = fr_pred[p], pa = fr_acc[p];
+    uint32_t cl = 0, ca = 0;
+    for (uint32_t q = 0; q < F; ++q) {
+      const uint32_t qp = fr_pred[q], qa = fr_acc[q];
+      cl += (qp < pp) || (qp == pp && q < p);
+      ca += (qa < pa) || (qa == pa && q < p);
+    }
+    rkL[p] = (uint16_t)cl;
+    rkA[p] = (uint16_t)ca;
+    thr_s[cl] = pp;
+    acc_s[ca] = (uint16_t)pa;
+  }
+  __syncthreads();
+  uint32_t *thr_g = reinterpret_cast<uint32_t *>(block + L.thr);
+  uint16_t *acc_g = reinterpret_cast<uint16_t *>(block + L.accs);
+  for (uint32_t i = tid; i < F; i += B) {
+    thr_g[i] = thr_s[i];
+    acc_g[i] = acc_s[i];
+  }
+  // bucket tables
+  const uint32_t acc_base = acc_s[0], acc_range = acc_s[F - 1] - acc_s[0];
+  uint32_t shift = 0;
+  while ((acc_range >> shift) > ACC_BUCKETS - 1) ++shift;
+  if (tid == 0) *meta_out = acc_base | (shift << 16);
+  unsigned char *startL = block + L.start, *startA = startL + SLO_BUCKET_BYTES;
+  for (uint32_t b = tid; b < SLO_BUCKET_BYTES + ACC_BUCKETS; b += B) {
+    uint32_t cnt = 0;
+    if (b < SLO_BUCKETS) {
+      if (b > 0) {
+        const uint32_t lo = slo_bucket_floor(b);       // every slo in the bucket is >= lo
+        for (uint32_t i = 0; i < F; ++i) cnt += thr_s[i] < lo;
+      }
+      startL[b] = (unsigned char)min(cnt, 255u);
+    } else if (b < SLO_BUCKET_BYTES) {
+      startL[b] = 0;
+    } else {
+      const uint32_t lo = acc_base + ((b - SLO_BUCKET_BYTES) << shift);   // every min_acc in the bucket is >= lo
+      for (uint32_t i = 0; i < F; ++i) cnt += acc_s[i] < lo;
+      startA[b - SLO_BUCKET_BYTES] = (unsigned char)min(cnt, 255u);
+    }
+  }
+  // masks
+  unsigned long long *ML = reinterpret_cast<unsigned long long *>(block + L.masks);
+  unsigned long long *MA = ML + (F + 1) * L.nw;
+  for (uint32_t idx = tid; idx < (F + 1) * L.nw; idx += B) {
+    const uint32_t r = idx / L.nw, w = idx - r * L.nw;
+    unsigned long long ml = 0, ma = 0;
+    const uint32_t p_end = min(F, 64u * w + 64u);
+    for (uint32_t p = 64u * w; p < p_end; ++p) {
+      const unsigned long long bit = 1ull << (p & 63u);
+      if (rkL[p] < r) ml |= bit;
+      if (rkA[p] >= r) ma |= bit;
+    }
+    ML[idx] = ml;
+    MA[idx] = ma;
+  }
+}
+
 __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long *k64 = reinterpret_cast<unsigned long long *>(smem_raw);   // cost<<32 | pred
   uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
+  unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
-  __shared__ uint32_t s_last;
+  __shared__ uint32_t s_last, s_total;
+  __shared__ uint32_t fr_pred[MASK_MAX_F], thr_s[MASK_MAX_F];
+  __shared__ uint16_t fr_acc[MASK_MAX_F], rkL[MASK_MAX_F], rkA[MASK_MAX_F], acc_s[MASK_MAX_F];
 
   const uint32_t t = blockIdx.x, tid = threadIdx.x, B = blockDim.x;
   const uint32_t base = c.task_off[t];
@@ -165,36 +240,50 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
     }
   }
 
-  // 3. prune + 4. compact.  In sorted order every dominator of p sits before p, and every
-  // earlier entry q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not
-  // larger by the sort, and it differs in some attribute or has the smaller id).
-  const uint32_t reg = c.reg_off[t];
+  // 3. prune.  In sorted order every dominator of p sits before p, and every earlier entry
+  // q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not larger by the
+  // sort, and it differs in some attribute or has the smaller id).
+  uint32_t my_kept = 0;
+  for (uint32_t p = tid; p < V; p += B) {
+    const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
+    bool kp = true;
+    for (uint32_t q = 0; q < p; ++q) {
+      if ((uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p) { kp = false; break; }
+    }
+    keep[p] = kp;
+    my_kept += kp;
+  }
+  if (tid == 0) s_total = 0;
+  __syncthreads();
+  my_kept = __reduce_add_sync(0xFFFFFFFFu, my_kept);
+  if ((tid & 31) == 0 && my_kept) atomicAdd(&s_total, my_kept);
+  __syncthreads();
+  const uint32_t F = s_total;
+  const BlockLayout L = block_layout(F);
+  unsigned char *block = c.regions + c.reg_off[t];
+
+  // 4. compact into the task block (scan order)
+  unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(block + L.keys);
+  uint32_t *ids_g = reinterpret_cast<uint32_t *>(block + L.ids);
   uint32_t kept_so_far = 0;
   for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
     const uint32_t p = p0 + tid;
-    bool keep = false;
-    uint32_t pred_p = 0, inv_p = 0, local = 0;
-    if (p < V) {
-      pred_p = (uint32_t)k64[p];
-      inv_p = k32[p] >> 16;
-      local = k32[p] & 0xFFFFu;
-      keep = true;
-      for (uint32_t q = 0; q < p; ++q) {
-        if ((uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p) { keep = false; break; }
-      }
-    }
+    const bool kp = p < V && keep[p];
     uint32_t total;
-    uint32_t off = block_excl_scan_flag(keep, warp_sums, total);
-    if (keep) {
-      const uint32_t acc = 10000u - inv_p;
-      c.f_key[reg + kept_so_far + off] = ((unsigned long long)acc << 32) | pred_p;
-      c.f_id[reg + kept_so_far + off] = c.s_id[base + local];
+    const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
+    if (kp) {
+      const uint32_t pred_p = (uint32_t)k64[p], acc = 10000u - (k32[p] >> 16);
+      keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
+      ids_g[pos] = c.s_id[base + (k32[p] & 0xFFFFu)];
+      if (L.nw) { fr_pred[pos] = pred_p; fr_acc[pos] = (uint16_t)acc; }
     }
     kept_so_far += total;
   }
-  if (tid == 0) c.f_len[t] = kept_so_far;
+  __syncthreads();
+  if (tid == 0) { c.f_len[t] = F; if (!L.nw) c.f_meta[t] = 0; }
+  if (L.nw) build_index(block, L, F, fr_pred, fr_acc, rkL, rkA, thr_s, acc_s, c.f_meta + t);
 
-  // 5. the CTA that finishes last packs all lists into the blob
+  // 5. the CTA that finishes last packs all blocks into the image
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -206,14 +295,17 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   __threadfence();
 
   const uint32_t T = c.n_tasks;
-  uint32_t *table = reinterpret_cast<uint32_t *>(c.blob);
-  // 5a. starts = exclusive prefix sum of the lengths (chunks of B tasks, running carry)
-  uint32_t carry = 0, longest = 0;
+  TaskDesc *desc = reinterpret_cast<TaskDesc *>(c.image);
+  const uint32_t desc_bytes = T * (uint32_t)sizeof(TaskDesc);
+  // 5a. block offsets = exclusive prefix sum of block sizes (chunks of B tasks, running carry)
+  uint32_t carry = desc_bytes, longest = 0, entries = 0, linear = 0;
   __shared__ uint32_t scan_buf[1024];
+  bool overflow = false;
   for (uint32_t t0 = 0; t0 < T; t0 += B) {
     const uint32_t tt = t0 + tid;
     const uint32_t len = tt < T ? __ldcg(c.f_len + tt) : 0u;
-    scan_buf[tid] = len;
+    const BlockLayout Lt = block_layout(len);
+    scan_buf[tid] = Lt.bytes;
     __syncthreads();
     for (uint32_t o = 1; o < B; o <<= 1) {      // Hillis-Steele inclusive scan
       uint32_t v = tid >= o ? scan_buf[tid - o] : 0u;
@@ -221,50 +313,58 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
       scan_buf[tid] += v;
       __syncthreads();
     }
-    if (tt < T) {
-      table[2 * tt] = carry + scan_buf[tid] - len;
-      table[2 * tt + 1] = len;
+    const uint32_t chunk_total = scan_buf[B - 1];
+    const uint32_t incl = scan_buf[tid];
+    __syncthreads();                                               // scan_buf is reused below
+    if (carry + chunk_total > c.image_capacity) overflow = true;   // uniform
+    if (tt < T && !overflow) {
+      const uint32_t off = carry + incl - Lt.bytes;
+      TaskDesc d;
+      d.off_masks = off + Lt.masks;
+      d.f_nw = len | (Lt.nw << 16);
+      d.acc_meta = __ldcg(c.f_meta + tt);
+      d.off_keys = off + Lt.keys;
+      d.off_thr = off + Lt.thr;
+      d.off_ids = off + Lt.ids;
+      d.off_accs = off + Lt.accs;
+      d.off_start = off + Lt.start;
+      desc[tt] = d;
+      // the block's offset, kept for the copy pass
+      scan_buf[tid] = off;
+    }
+    __syncthreads();
+    // 5b. copy this chunk's blocks (one warp per task, 16 bytes per lane and step)
+    if (!overflow) {
+      const uint32_t lane = tid & 31, warp = tid >> 5, nwarps = B >> 5;
+      for (uint32_t i = warp; i < B && t0 + i < T; i += nwarps) {
+        const uint32_t len_i = __ldcg(c.f_len + t0 + i);
+        const uint32_t bytes_i = block_layout(len_i).bytes;
+        const uint4 *src = reinterpret_cast<const uint4 *>(c.regions + c.reg_off[t0 + i]);
+        uint4 *dst = reinterpret_cast<uint4 *>(c.image + scan_buf[i]);
+        for (uint32_t e = lane; e < (bytes_i >> 4); e += 32) dst[e] = __ldcg(src + e);
+      }
     }
     longest = max(longest, len);
-    const uint32_t chunk_total = scan_buf[B - 1];
+    entries += len;
+    linear += (len > 0 && Lt.nw == 0);
     __syncthreads();
     carry += chunk_total;
   }
-  if (tid == 0 && (T & 1u)) { table[2 * T] = 0; table[2 * T + 1] = 0; }   // pad entry
-  const uint32_t E = carry;
-  const uint32_t E_pad = (E + 3u) & ~3u;
-  const uint32_t bytes = blob_total_bytes(c.n_tasks_pad, E_pad);
-  if (bytes > c.blob_capacity) {
-    if (tid == 0) { atomicMax(c.err, (uint32_t)DEV_ERR_BLOB_OVERFLOW); *c.done_ctr = 0; }
-    return;
-  }
-  __syncthreads();   // table writes visible to the CTA
-  unsigned long long *bkeys = reinterpret_cast<unsigned long long *>(c.blob + blob_table_bytes(c.n_tasks_pad));
-  uint32_t *bids = reinterpret_cast<uint32_t *>(bkeys + E_pad);
-  // 5b. one warp per task copies its list
-  const uint32_t lane = tid & 31, warp = tid >> 5, nw = B >> 5;
-  for (uint32_t tt = warp; tt < T; tt += nw) {
-    const uint32_t start = table[2 * tt], len = table[2 * tt + 1], r = c.reg_off[tt];
-    for (uint32_t e = lane; e < len; e += 32) {
-      bkeys[start + e] = __ldcg(c.f_key + r + e);
-      bids[start + e] = __ldcg(c.f_id + r + e);
-    }
-  }
-  for (uint32_t e = E + tid; e < E_pad; e += B) {   // padding never matches a query
-    bkeys[e] = 0xFFFFFFFFull;                        // pred = 2^32-1, acc = 0
-    bids[e] = INFAAS_INVALID;
-  }
-  // longest list (for reporting)
+  // totals for reporting
   longest = __reduce_max_sync(0xFFFFFFFFu, longest);
-  if (lane == 0) warp_sums[warp] = longest;
+  entries = __reduce_add_sync(0xFFFFFFFFu, entries);
+  linear = __reduce_add_sync(0xFFFFFFFFu, linear);
+  __shared__ uint32_t tot[3];
+  if (tid == 0) tot[0] = tot[1] = tot[2] = 0;
+  __syncthreads();
+  if ((tid & 31) == 0) { atomicMax(&tot[0], longest); atomicAdd(&tot[1], entries); atomicAdd(&tot[2], linear); }
   __syncthreads();
   if (tid == 0) {
-    uint32_t m = 0;
-    for (uint32_t w = 0; w < nw; ++w) m = max(m, warp_sums[w]);
-    c.blob_hdr[0] = bytes;
-    c.blob_hdr[1] = E_pad;
-    c.blob_hdr[2] = m;
-    c.blob_hdr[3] = E;
+    if (overflow) atomicMax(c.err, (uint32_t)DEV_ERR_IMAGE_OVERFLOW);
+    c.image_hdr[0] = overflow ? 0xFFFFFFFFu : carry;
+    c.image_hdr[1] = tot[0];
+    c.image_hdr[2] = tot[1];
+    c.image_hdr[3] = tot[2];
     *c.done_ctr = 0;
   }
 }
@@ -289,8 +389,8 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream) {
   uint32_t P = 1;
   while (P < c.max_task_variants) P <<= 1;
-  uint32_t block = P < 64 ? 64 : (P > 1024 ? 1024 : P);
-  size_t smem = (size_t)P * 12;
+  uint32_t block = P < 128 ? 128 : (P > 1024 ? 1024 : P);
+  size_t smem = (size_t)P * 13;
   rebuild_kernel<<<c.n_tasks, block, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
   return cudaGetLastError();
 }
