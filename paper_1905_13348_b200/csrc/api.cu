@@ -118,7 +118,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   std::vector<uint32_t> reg_off(n_tasks + 1, 0);
   uint64_t region_bytes = 0;
   for (uint32_t t = 0; t < n_tasks; ++t) {
-    region_bytes += infaas::block_capacity(task_off[t + 1] - task_off[t]);
+    region_bytes += infaas::region_capacity(task_off[t + 1] - task_off[t]);
     if (region_bytes > 0xF0000000ull) return INFAAS_E_TOO_LARGE;
     reg_off[t + 1] = (uint32_t)region_bytes;
   }
@@ -143,7 +143,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   if (scope.status != cudaSuccess) { delete c; return cuda_fail(scope.status); }
 
   // ---- one arena, carved into 256-byte aligned arrays ----
-  const uint64_t worst_image = (uint64_t)n_tasks * sizeof(infaas::TaskDesc) + region_bytes;
+  uint64_t worst_image = infaas::image_var_offset(n_tasks);
+  for (uint32_t t = 0; t < n_tasks; ++t) worst_image += infaas::var_capacity(task_off[t + 1] - task_off[t]);
   if (worst_image > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
   size_t total = 0;
   auto carve = [&total](size_t bytes) { size_t off = total; total += round_up(bytes, 256); return off; };
@@ -154,7 +155,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
   const size_t o_regions = carve((size_t)region_bytes);
-  const size_t o_flen = carve((size_t)n_tasks * 4), o_fmeta = carve((size_t)n_tasks * 4);
+  const size_t o_flen = carve((size_t)n_tasks * 4), o_fks = carve((size_t)n_tasks * 4);
+  const size_t o_fvar = carve((size_t)n_tasks * 4), o_fhdr = carve((size_t)n_tasks * 8);
   const size_t o_image = carve((size_t)worst_image), o_hdr = carve(16);
   const size_t o_counters = carve(24), o_done = carve(4), o_err = carve(4);
 
@@ -196,7 +198,9 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.count_by_id = reinterpret_cast<uint32_t *>(base + o_count);
   d.regions = base + o_regions;
   d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
-  d.f_meta = reinterpret_cast<uint32_t *>(base + o_fmeta);
+  d.f_ks = reinterpret_cast<uint32_t *>(base + o_fks);
+  d.f_var_bytes = reinterpret_cast<uint32_t *>(base + o_fvar);
+  d.f_hdr = reinterpret_cast<infaas::TaskHdr *>(base + o_fhdr);
   d.image = base + o_image;
   d.image_capacity = (uint32_t)worst_image;
   d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
@@ -307,7 +311,8 @@ int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_id
   *h_len = len;
   const uint32_t ncopy = len < cap ? len : cap;
   if (h_ids && ncopy) {
-    const unsigned char *ids = c->d.regions + c->reg_off[task] + infaas::block_layout(len).ids;
+    const uint32_t V = c->task_off[task + 1] - c->task_off[task];
+    const unsigned char *ids = c->d.regions + c->reg_off[task] + 8u * (size_t)V;
     CUDA_TRY(cudaMemcpyAsync(h_ids, ids, (size_t)ncopy * 4, cudaMemcpyDeviceToHost, s));
     CUDA_TRY(cudaStreamSynchronize(s));
   }

@@ -14,71 +14,62 @@ namespace infaas {
 // Scan list of a task: its non-dominated variants sorted by (cost, pred_lat, 10000-acc, id).
 // Position p in that order is what selection returns the smallest feasible of.
 //
-// Task block (one per task, 16-byte aligned, self-contained).  For a list of F entries:
-//     keys   u64[F]   pred_lat (bits 0..31) | acc_bp (bits 32..47), scan order
-//     ids    u32[F]   variant ids, scan order
-//   and, if F <= MASK_MAX_F (the "indexed" form, nw = ceil(F/64) mask words):
-//     thr    u32[F]   pred_lat ascending
-//     accs   u16[F]   acc_bp ascending                      (padded to 4 bytes)
-//     startL u8[260]  per SLO bucket: lower bound of #{thr <= slo}   (257 used)
-//     startA u8[128]  per accuracy bucket: lower bound of #{accs < min_acc}
-//     ML     u64[(F+1)*nw]   ML[r] = positions whose pred_lat is among the r smallest
-//     MA     u64[(F+1)*nw]   MA[k] = positions whose acc_bp is NOT among the k smallest
-//   A query with r = #{thr <= slo} and k = #{accs < min_acc} is met exactly by the
-//   positions in ML[r] & MA[k]; the answer is the lowest set bit.
-//   SLO bucket of s: 0 for s = 0, else 1 + (eighth-octave index of s) -- the top 11 bits
-//   of s converted to float (round toward zero), minus 1015.
-//   Accuracy bucket of m: min(127, max(0, m - acc_base) >> acc_shift).
+// For a list of F <= INDEX_MAX_F entries the rebuild kernel derives an exact index:
+//   Pd[0..Ks)  distinct pred_lat values ascending,  Ad[0..Ka)  distinct acc_bp ascending,
+//   r(slo) = #{Pd <= slo},  k(min_acc) = #{Ad < min_acc},
+//   T2[r][k] = first position whose pred_lat is among the r smallest values and whose
+//              acc_bp is not among the k smallest values (0xFF: none) -- the answer.
+// r comes from a table of SLO_BUCKETS records indexed by a monotone bucket of slo (top bits
+// of slo converted to float, shifted by `sh`, relative to `bmin`); a record holds the rank
+// below the bucket and the one distinct value inside it (as a 24-bit offset from the
+// bucket's smallest slo); buckets with two or more values are flagged and such queries take
+// the exact slow path.  k comes from a bitmap over acc values with running popcounts (24
+// bitmap bits + 8 prefix bits per word), exact at one basis point.
 //
-// Image: TaskDesc[n_tasks] followed by the blocks back to back; this is what the
-// selection kernel stages in shared memory.  All offsets in a TaskDesc are bytes from the
-// start of the image.
+// Image (what the selection kernel stages in shared memory), all parts 64-byte aligned:
+//   hdr   u64[n_tasks]            per-task packed parameters (TaskHdr below)
+//   slo   u32[n_tasks][SLO_BUCKETS]   SLO records: lb << 24 | delta ; lb == 0xFF: flagged
+//   var   per-task blocks back to back, each: ids u32[8*Fp8], acc bitmap u32[nbw],
+//         T2 u8[(Ks+1)*width], padded to 64 bytes
+//
+// Cold data (read from global memory by the slow path only), per task in its region, V =
+// number of the task's variants:
+//   keys u64[V] (F used)  pred_lat | acc_bp << 32 in scan order;  ids u32[V] (F used);
+//   Pd u32[Ks];  then, 64-byte aligned, the var block before it is packed into the image
 // ---------------------------------------------------------------------------------------
-constexpr uint32_t MASK_MAX_F = 256;
-constexpr uint32_t SLO_BUCKETS = 257;
-constexpr uint32_t SLO_BUCKET_BYTES = 260;
-constexpr uint32_t ACC_BUCKETS = 128;
-constexpr uint32_t SLO_BUCKET_BIAS = 1015;   // (127 << 3) - 1: float exponent of 1.0, three mantissa bits
+constexpr uint32_t INDEX_MAX_F = 248;
+constexpr uint32_t SLO_BUCKETS = 256;
+constexpr uint32_t ACC_WORD_BITS = 24;
+constexpr uint32_t MAX_ACC_WORDS = 420;          // covers 0..10000 bp at 24 per word
+constexpr uint32_t SLO_FLAGGED = 0xFFu;
+constexpr uint32_t VB_NOT_INDEXED = 0xFFEu;      // hdr.var_base value: list too long for the index
+constexpr uint32_t VB_NO_VARIANTS = 0xFFFu;      // hdr.var_base value: the task has no variant
 
-struct __align__(16) TaskDesc {   // 32 bytes
-  uint32_t off_masks;   // ML; MA follows (F+1)*nw words later
-  uint32_t f_nw;        // F | nw << 16 ; nw == 0: not indexed (linear scan)
-  uint32_t acc_meta;    // acc_base | acc_shift << 16
-  uint32_t off_keys;
-  uint32_t off_thr;
-  uint32_t off_ids;
-  uint32_t off_accs;
-  uint32_t off_start;   // startL; startA is SLO_BUCKET_BYTES further
+// hdr word 0: var_base (12 bits, units of 64 B from the start of the var section)
+//             | acc_min4 << 12 (12 bits, units of 4 bp) | sh << 24 (3 bits) | Fp8 << 27 (5 bits)
+// hdr word 1: bmin (15 bits) | nbw << 15 (9 bits) | width2 << 24 (7 bits, units of 2)
+struct TaskHdr {
+  uint32_t w0, w1;
 };
 
-struct BlockLayout {    // byte offsets inside a task block
-  uint32_t keys, ids, thr, accs, start, masks, bytes, nw;
-};
+inline __host__ __device__ uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-inline __host__ __device__ BlockLayout block_layout(uint32_t F) {
-  BlockLayout L;
-  L.nw = (F > 0 && F <= MASK_MAX_F) ? (F + 63u) / 64u : 0u;
-  L.keys = 0;
-  L.ids = 8u * F;
-  uint32_t end = 12u * F;
-  L.thr = L.accs = L.start = L.masks = end;
-  if (L.nw) {
-    L.thr = end;
-    L.accs = L.thr + 4u * F;
-    L.start = L.accs + ((2u * F + 3u) & ~3u);
-    L.masks = (L.start + SLO_BUCKET_BYTES + ACC_BUCKETS + 7u) & ~7u;
-    end = L.masks + 16u * (F + 1u) * L.nw;
-  }
-  L.bytes = (end + 15u) & ~15u;
-  return L;
+inline __host__ __device__ uint32_t image_slo_offset(uint32_t n_tasks) { return round_up_u32(8u * n_tasks, 64u); }
+inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) {
+  return image_slo_offset(n_tasks) + 4u * SLO_BUCKETS * n_tasks;
 }
 
-// Largest block a task with V variants can need (every variant non-dominated, or the
-// longest indexed list, whichever is larger).
-inline __host__ __device__ uint32_t block_capacity(uint32_t V) {
-  uint32_t a = block_layout(V).bytes;
-  uint32_t b = block_layout(V < MASK_MAX_F ? V : MASK_MAX_F).bytes;
-  return a > b ? a : b;
+// Worst-case bytes of one task's var block and of its region (cold data + var block).
+inline __host__ __device__ uint32_t var_capacity(uint32_t V) {
+  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
+  return round_up_u32(4u * MAX_ACC_WORDS + 4u * round_up_u32(F, 8) + (F + 1u) * (F + 2u), 64u);
+}
+inline __host__ __device__ uint32_t region_var_offset(uint32_t V) {
+  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
+  return round_up_u32(12u * V + 4u * F, 64u);     // after keys[V], ids[V] and Pd[min(V, INDEX_MAX_F)]
+}
+inline __host__ __device__ uint32_t region_capacity(uint32_t V) {
+  return region_var_offset(V) + var_capacity(V);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -91,7 +82,7 @@ struct DeviceCatalog {
   uint32_t max_task_variants;
 
   const uint32_t *task_off;  // [n_tasks + 1]
-  const uint32_t *reg_off;   // [n_tasks + 1] byte offset of each task's block region
+  const uint32_t *reg_off;   // [n_tasks + 1] byte offset of each task's region
   const uint32_t *s_lat;
   const uint16_t *s_batch;
   const uint16_t *s_acc;
@@ -102,11 +93,13 @@ struct DeviceCatalog {
   unsigned long long *s_served;
   uint32_t *count_by_id;     // [n_variants], zero between windows
 
-  unsigned char *regions;    // task blocks at their worst-case offsets (16-byte aligned)
+  unsigned char *regions;    // per task: keys, Pd, then the var block before packing
   uint32_t *f_len;           // [n_tasks] list length F
-  uint32_t *f_meta;          // [n_tasks] acc_base | acc_shift << 16
+  uint32_t *f_ks;            // [n_tasks] number of distinct pred_lat values (0 if not indexed)
+  uint32_t *f_var_bytes;     // [n_tasks] bytes of the task's var block (0 if not indexed)
+  TaskHdr *f_hdr;            // [n_tasks] header words without var_base (filled in when packing)
 
-  unsigned char *image;      // packed image, image_capacity bytes, 16-byte aligned
+  unsigned char *image;      // packed image, image_capacity bytes, 256-byte aligned
   uint32_t image_capacity;
   uint32_t *image_hdr;       // [4]: bytes, longest list, total entries, tasks not indexed
 

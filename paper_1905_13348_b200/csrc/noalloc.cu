@@ -39,7 +39,9 @@ extern "C" int infaas_tally_static(const uint32_t *d_decision, uint64_t n, uint3
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_scratch_addr[cuda_device]) {
       void *p = nullptr;
-      if (cudaGetSymbolAddress(&p, g_tally_scratch) != cudaSuccess || !p) rc = INFAAS_E_CUDA;
+      // (the tally kernels' shared-memory limit is a per-device attribute, set here too)
+      if (cudaGetSymbolAddress(&p, g_tally_scratch) != cudaSuccess || !p ||
+          infaas::prepare_rebuild_kernel() != cudaSuccess) rc = INFAAS_E_CUDA;
       else g_scratch_addr[cuda_device] = static_cast<StaticScratch *>(p);
     }
     scratch = g_scratch_addr[cuda_device];

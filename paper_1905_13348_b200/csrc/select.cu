@@ -6,14 +6,15 @@
 // Each task's scan list is sorted by (cost, pred_lat, -acc, id) and pruned to non-dominated
 // variants, so the answer for a feasible query is the FIRST list position that meets both
 // requirements.  Instead of walking the list, a thread ranks the query's SLO among the
-// list's latencies and its minimum accuracy among the list's accuracies (bucket table +
-// a short refine loop) and ANDs two precomputed position bitmasks; the lowest set bit is
-// the answer (layout in common.cuh).  The packed image of all tasks is staged in shared
-// memory once per CTA with bulk asynchronous copies (TMA, mbarrier completion); queries
-// stream through with 128-bit loads and stores, four per thread and iteration.
-// Queries without a feasible variant (a few percent) are parked in a per-warp list and
-// resolved 32 at a time with all lanes busy: a pass over the list computing the distance
-// d = 10^4 * over_lat + slo * under_acc.
+// list's distinct latencies (one bucket record, one comparison) and its minimum accuracy
+// among the list's distinct accuracies (one bitmap word, one popcount) and reads the
+// answer's position from a small per-task table indexed by the two ranks (layout in
+// common.cuh): five shared-memory loads per query, no loop.  The packed image of all
+// tasks is staged in shared memory once per CTA with bulk asynchronous copies (TMA,
+// mbarrier completion); queries stream through with 128-bit loads and stores, four per
+// thread and iteration.  Queries that need more (no feasible variant, a flagged SLO bucket,
+// a task whose list is too long for the index) are parked in a per-warp list and resolved
+// exactly 32 at a time with all lanes busy.
 #include "common.cuh"
 
 namespace infaas {
@@ -72,94 +73,117 @@ __device__ __forceinline__ bool stage_image(unsigned char *dst, const unsigned c
 struct SharedImage {
   uint32_t base;
   __device__ __forceinline__ uint32_t u8(uint32_t off) const {
-    uint32_t v; asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
-  }
-  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
-    uint32_t v; asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
+    uint32_t v; asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
   }
   __device__ __forceinline__ uint32_t u32(uint32_t off) const {
-    uint32_t v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
+    uint32_t v; asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
   }
-  __device__ __forceinline__ unsigned long long u64(uint32_t off) const {
-    unsigned long long v; asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(base + off)); return v;
-  }
-  __device__ __forceinline__ uint4 v4(uint32_t off) const {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(base + off));
-    return v;
+  __device__ __forceinline__ uint2 v2(uint32_t off) const {
+    uint2 v; asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(base + off)); return v;
   }
 };
 
 struct GlobalImage {
   const unsigned char *base;
   __device__ __forceinline__ uint32_t u8(uint32_t off) const { return __ldg(base + off); }
-  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
-    return __ldg(reinterpret_cast<const uint16_t *>(base + off));
-  }
   __device__ __forceinline__ uint32_t u32(uint32_t off) const {
     return __ldg(reinterpret_cast<const uint32_t *>(base + off));
   }
-  __device__ __forceinline__ unsigned long long u64(uint32_t off) const {
-    return __ldg(reinterpret_cast<const unsigned long long *>(base + off));
-  }
-  __device__ __forceinline__ uint4 v4(uint32_t off) const {
-    return __ldg(reinterpret_cast<const uint4 *>(base + off));
+  __device__ __forceinline__ uint2 v2(uint32_t off) const {
+    return __ldg(reinterpret_cast<const uint2 *>(base + off));
   }
 };
 
-// First list position that meets (slo, min_acc), as a decision; PENDING if none does.
-template <class Img>
-__device__ __forceinline__ uint32_t decide(const Img &img, uint32_t n_tasks, uint32_t task,
-                                           uint32_t slo, uint32_t min_acc) {
-  if (task >= n_tasks) return INFAAS_INVALID;
-  const uint4 d0 = img.v4(task * 32u);        // off_masks, f_nw, acc_meta, off_keys
-  const uint4 d1 = img.v4(task * 32u + 16u);  // off_thr, off_ids, off_accs, off_start
-  const uint32_t F = d0.y & 0xFFFFu, nw = d0.y >> 16;
-  if (F == 0) return INFAAS_INVALID;
-  if (nw == 0) {   // list too long for the index: walk it
-    for (uint32_t i = 0; i < F; ++i) {
-      const unsigned long long e = img.u64(d0.w + 8u * i);
-      if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return img.u32(d1.y + 4u * i);
-    }
-    return PENDING;
-  }
-  // r = #{list latencies <= slo}
-  const uint32_t fb = __float_as_uint(__uint2float_rz(slo)) >> 20;
-  uint32_t r = img.u8(d1.w + max(fb, SLO_BUCKET_BIAS) - SLO_BUCKET_BIAS);
-  while (r < F && img.u32(d1.x + 4u * r) <= slo) ++r;
-  // k = #{list accuracies < min_acc}
-  const uint32_t acc_base = d0.z & 0xFFFFu, acc_shift = d0.z >> 16;
-  const uint32_t above = min_acc > acc_base ? min_acc - acc_base : 0u;
-  uint32_t k = img.u8(d1.w + SLO_BUCKET_BYTES + min(above >> acc_shift, ACC_BUCKETS - 1u));
-  while (k < F && img.u16(d1.z + 2u * k) < min_acc) ++k;
-  // positions that meet both = ML[r] & MA[k]
-  const uint32_t ml = d0.x + 8u * r * nw, ma = d0.x + 8u * ((F + 1u) * nw + k * nw);
-  for (uint32_t w = 0; w < nw; ++w) {
-    const unsigned long long x = img.u64(ml + 8u * w) & img.u64(ma + 8u * w);
-    if (x) return img.u32(d1.y + 4u * (64u * w + (uint32_t)__ffsll((long long)x) - 1u));
-  }
-  return PENDING;
+// Per-task parameters unpacked from the two header words (see common.cuh).
+struct TaskParams {
+  uint32_t vb, acc_min, sh, ids_off, bitmap_off, t2_off, bmin, nbw, width;
+};
+__device__ __forceinline__ TaskParams unpack_hdr(uint32_t w0, uint32_t w1, uint32_t var0) {
+  TaskParams P;
+  P.vb = w0 & 0xFFFu;
+  P.acc_min = ((w0 >> 12) & 0xFFFu) << 2;
+  P.sh = (w0 >> 24) & 7u;
+  P.bmin = w1 & 0x7FFFu;
+  P.nbw = (w1 >> 15) & 0x1FFu;
+  P.width = ((w1 >> 24) & 0x7Fu) << 1;
+  P.ids_off = var0 + (P.vb << 6);
+  P.bitmap_off = P.ids_off + ((w0 >> 27) << 5);
+  P.t2_off = P.bitmap_off + (P.nbw << 2);
+  return P;
 }
 
-// Nearest miss of a query no list entry meets: d = 10^4 * over_lat + slo * under_acc
-// (64-bit); strict '<' keeps the first of equal distances, i.e. the smallest
-// (cost, pred_lat, -acc, id).
+// k = #{distinct list accuracies < min_acc}, from the bitmap with running popcounts.
 template <class Img>
-__device__ __forceinline__ uint32_t nearest_miss(const Img &img, uint32_t task, uint32_t slo,
-                                                 uint32_t min_acc) {
-  const uint4 d0 = img.v4(task * 32u);
-  const uint32_t F = d0.y & 0xFFFFu, off_ids = img.u32(task * 32u + 20u);
+__device__ __forceinline__ uint32_t acc_rank(const Img &img, const TaskParams &P, uint32_t min_acc) {
+  const uint32_t x = min(max(min_acc, P.acc_min) - P.acc_min, ACC_WORD_BITS * P.nbw - 1u);
+  const uint32_t w = (x * 43691u) >> 20;                    // x / 24 for x < 2^16
+  const uint32_t word = img.u32(P.bitmap_off + (w << 2));
+  return (word >> 24) + __popc(word & ((1u << (x - w * ACC_WORD_BITS)) - 1u));
+}
+
+// Fast path, no loops: the decision, INFAAS_INVALID, or PENDING when the query has to take
+// the exact slow path (flagged SLO bucket, task without index) or nothing is feasible.
+template <class Img>
+__device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks, uint32_t slo_off,
+                                                uint32_t var0, uint32_t task, uint32_t slo,
+                                                uint32_t min_acc) {
+  if (task >= n_tasks) return INFAAS_INVALID;
+  const uint2 h = img.v2(task << 3);
+  const TaskParams P = unpack_hdr(h.x, h.y, var0);
+  if (P.vb >= VB_NOT_INDEXED) return P.vb == VB_NO_VARIANTS ? INFAAS_INVALID : PENDING;
+  // r = #{distinct list latencies <= slo}: bucket record + one comparison
+  const uint32_t b = (__float_as_uint(__uint2float_rz(slo)) >> 16) >> P.sh;
+  const uint32_t j = min(max(b, P.bmin) - P.bmin, SLO_BUCKETS - 1u);
+  const uint32_t lo = j ? __float2uint_ru(__uint_as_float(((P.bmin + j) << P.sh) << 16)) : 0u;
+  const uint32_t rec = img.u32(slo_off + ((task * SLO_BUCKETS + j) << 2));
+  const uint32_t lb = rec >> 24;
+  const uint32_t r = lb == SLO_FLAGGED ? 0u : lb + ((slo - lo) >= (rec & 0x00FFFFFFu));
+  const uint32_t k = acc_rank(img, P, min_acc);
+  const uint32_t pos = img.u8(P.t2_off + r * P.width + k);
+  if (lb == SLO_FLAGGED || pos == 0xFFu) return PENDING;
+  return img.u32(P.ids_off + (pos << 2));
+}
+
+// Exact slow path for a parked query: the decision, or the nearest miss when nothing is
+// feasible: d = 10^4 * over_lat + slo * under_acc (64-bit); strict '<' keeps the first of
+// equal distances, i.e. the smallest (cost, pred_lat, -acc, id).  Cold data comes from the
+// task's region in global memory.
+template <class Img>
+__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t var0,
+                                                uint32_t task, uint32_t slo, uint32_t min_acc) {
+  const uint32_t F = __ldg(c.f_len + task), Ks = __ldg(c.f_ks + task);
+  const uint32_t V = __ldg(c.task_off + task + 1) - __ldg(c.task_off + task);
+  const unsigned char *region = c.regions + __ldg(c.reg_off + task);
+  const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(region);
+  const uint32_t *ids = reinterpret_cast<const uint32_t *>(region + 8u * V);
+  const uint2 h = img.v2(task << 3);
+  const TaskParams P = unpack_hdr(h.x, h.y, var0);
+  if (P.vb < VB_NOT_INDEXED) {
+    const uint32_t *Pd = reinterpret_cast<const uint32_t *>(region + 12u * V);
+    uint32_t lo = 0, hi = Ks;                          // r = #{Pd <= slo}
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (__ldg(Pd + mid) <= slo) lo = mid + 1; else hi = mid;
+    }
+    const uint32_t pos = img.u8(P.t2_off + lo * P.width + acc_rank(img, P, min_acc));
+    if (pos != 0xFFu) return __ldg(ids + pos);
+  } else {
+    for (uint32_t i = 0; i < F; ++i) {
+      const unsigned long long e = __ldg(keys + i);
+      if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return __ldg(ids + i);
+    }
+  }
   unsigned long long best = ~0ull;
   uint32_t best_i = 0;
   for (uint32_t i = 0; i < F; ++i) {
-    const unsigned long long e = img.u64(d0.w + 8u * i);
+    const unsigned long long e = __ldg(keys + i);
     const uint32_t pred = (uint32_t)e, acc = (uint32_t)(e >> 32);
     const uint32_t over = pred > slo ? pred - slo : 0u;
     const uint32_t under = min_acc > acc ? min_acc - acc : 0u;
     const unsigned long long d = (unsigned long long)over * 10000ull + (unsigned long long)slo * under;
     if (d < best) { best = d; best_i = i; }
   }
-  return INFAAS_NO_FEASIBLE | img.u32(off_ids + 4u * best_i);
+  return INFAAS_NO_FEASIBLE | __ldg(ids + best_i);
 }
 
 struct Queries {
@@ -171,12 +195,13 @@ struct Queries {
 
 // Resolve up to 32 parked queries, one per lane.  `rel` is the query's offset from `q0`.
 template <class Img>
-__device__ __forceinline__ void resolve_parked(const Img &img, const Queries &q, uint64_t q0,
-                                               const uint32_t *park, uint32_t first, uint32_t count) {
+__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, uint32_t var0,
+                                               const Queries &q, uint64_t q0, const uint32_t *park,
+                                               uint32_t first, uint32_t count) {
   const uint32_t lane = threadIdx.x & 31;
   if (lane < count) {
     const uint64_t i = q0 + park[first + lane];
-    q.decision[i] = nearest_miss(img, q.task[i], q.slo[i], q.min_acc[i]);
+    q.decision[i] = decide_slow(img, c, var0, q.task[i], q.slo[i], q.min_acc[i]);
   }
 }
 
@@ -188,8 +213,10 @@ __device__ __forceinline__ void park_append(uint32_t *park, uint32_t &cnt, bool 
 }
 
 template <class Img>
-__device__ __forceinline__ void select_body(const Img &img, uint32_t n_tasks, const Queries &q,
+__device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
                                             uint64_t n, uint64_t per_cta, uint32_t *park_all) {
+  const uint32_t n_tasks = c.n_tasks;
+  const uint32_t slo_off = image_slo_offset(n_tasks), var0 = image_var_offset(n_tasks);
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t *park = park_all + warp * PARK_CAP;
   uint32_t parked = 0;
@@ -220,10 +247,10 @@ __device__ __forceinline__ void select_body(const Img &img, uint32_t n_tasks, co
       a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
     }
     uint4 d;
-    d.x = decide(img, n_tasks, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
-    d.y = decide(img, n_tasks, t.x >> 16, s.y, a.x >> 16);
-    d.z = decide(img, n_tasks, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
-    d.w = decide(img, n_tasks, t.y >> 16, s.w, a.y >> 16);
+    d.x = decide_fast(img, n_tasks, slo_off, var0, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
+    d.y = decide_fast(img, n_tasks, slo_off, var0, t.x >> 16, s.y, a.x >> 16);
+    d.z = decide_fast(img, n_tasks, slo_off, var0, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
+    d.w = decide_fast(img, n_tasks, slo_off, var0, t.y >> 16, s.w, a.y >> 16);
     const uint32_t rel = (uint32_t)(tile * WARP_TILE) + lane * 4u;
     uint32_t *out = q.decision + q0 + rel;
     const bool any_pending = d.x == PENDING || d.y == PENDING || d.z == PENDING || d.w == PENDING;
@@ -243,7 +270,7 @@ __device__ __forceinline__ void select_body(const Img &img, uint32_t n_tasks, co
       __syncwarp();
       while (parked >= 32) {
         parked -= 32;
-        resolve_parked(img, q, q0, park, parked, 32);
+        resolve_parked(img, c, var0, q, q0, park, parked, 32);
       }
       __syncwarp();
     }
@@ -256,7 +283,7 @@ __device__ __forceinline__ void select_body(const Img &img, uint32_t n_tasks, co
       uint32_t d = 0;
       if (rel < span) {
         const uint64_t i = q0 + rel;
-        d = decide(img, n_tasks, q.task[i], q.slo[i], q.min_acc[i]);
+        d = decide_fast(img, n_tasks, slo_off, var0, q.task[i], q.slo[i], q.min_acc[i]);
         if (d != PENDING) q.decision[i] = d;
       }
       park_append(park, parked, rel < span && d == PENDING, (uint32_t)rel);
@@ -264,33 +291,31 @@ __device__ __forceinline__ void select_body(const Img &img, uint32_t n_tasks, co
     __syncwarp();
     while (parked >= 32) {
       parked -= 32;
-      resolve_parked(img, q, q0, park, parked, 32);
+      resolve_parked(img, c, var0, q, q0, park, parked, 32);
     }
   }
   __syncwarp();
-  resolve_parked(img, q, q0, park, 0, parked);
+  resolve_parked(img, c, var0, q, q0, park, 0, parked);
 }
 
 __global__ void __launch_bounds__(SELECT_THREADS, 1)
-select_kernel(const unsigned char *__restrict__ image, const uint32_t *__restrict__ image_hdr,
-              uint32_t n_tasks, uint32_t image_smem, Queries q, uint64_t n, uint64_t per_cta,
-              uint32_t *err) {
+select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint64_t per_cta) {
   extern __shared__ __align__(128) unsigned char smem[];   // [park lists][staged image]
   __shared__ __align__(8) unsigned long long mbar;
   uint32_t *park = reinterpret_cast<uint32_t *>(smem);
   unsigned char *staged = smem + PARK_BYTES;
-  const uint32_t bytes = image_hdr[0];
+  const uint32_t bytes = c.image_hdr[0];
   if (bytes <= image_smem) {
-    if (!stage_image(staged, image, bytes, &mbar)) {
-      if (threadIdx.x == 0) atomicMax(err, (uint32_t)DEV_ERR_STAGE_TIMEOUT);
+    if (!stage_image(staged, c.image, bytes, &mbar)) {
+      if (threadIdx.x == 0) atomicMax(c.err, (uint32_t)DEV_ERR_STAGE_TIMEOUT);
       return;
     }
     SharedImage img{smem_u32(staged)};
-    select_body(img, n_tasks, q, n, per_cta, park);
+    select_body(img, c, q, n, per_cta, park);
   } else {
     // the image does not fit in shared memory: read it from global memory (L1/L2 resident)
-    GlobalImage img{image};
-    select_body(img, n_tasks, q, n, per_cta, park);
+    GlobalImage img{c.image};
+    select_body(img, c, q, n, per_cta, park);
   }
 }
 
@@ -314,8 +339,8 @@ cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const 
   if (per_cta > 0xFFFFFFFFull) return cudaErrorInvalidValue;
   grid = (n + per_cta - 1) / per_cta;
   Queries q{d_task, d_slo, d_min_acc, d_decision};
-  select_kernel<<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(
-      c.image, c.image_hdr, c.n_tasks, image_smem, q, n, per_cta, c.err);
+  select_kernel<<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n,
+                                                                                     per_cta);
   return cudaGetLastError();
 }
 

@@ -72,6 +72,49 @@ tally_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_varia
   if (threadIdx.x < 3 && blk[threadIdx.x]) atomicAdd(&counters[threadIdx.x], (unsigned long long)blk[threadIdx.x]);
 }
 
+// Same tallies with a private histogram per CTA in shared memory (one u32 bin per variant):
+// shared-memory atomics absorb the hot variants, and each CTA adds only its non-zero bins
+// to the global counts at the end.  Used when the bins fit and the batch is large.
+constexpr int TALLY_SMEM_THREADS = 512;
+
+__global__ void __launch_bounds__(TALLY_SMEM_THREADS)
+tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_variants,
+                  uint32_t *__restrict__ count_by_id, unsigned long long *__restrict__ counters) {
+  extern __shared__ uint32_t hist[];
+  __shared__ uint32_t blk[3];
+  for (uint32_t i = threadIdx.x; i < n_variants; i += blockDim.x) hist[i] = 0;
+  if (threadIdx.x < 3) blk[threadIdx.x] = 0;
+  __syncthreads();
+  uint32_t n_feas = 0, n_nofeas = 0, n_inval = 0;
+  auto one = [&](uint32_t d) {
+    if (d < n_variants) { atomicAdd(&hist[d], 1u); ++n_feas; }   // d < n_variants < 2^31: bit 31 clear
+    else if (d != INFAAS_INVALID && (d & INFAAS_NO_FEASIBLE)) ++n_nofeas;
+    else ++n_inval;
+  };
+  const uint64_t n4 = n >> 2;
+  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  const uint4 *dec4 = reinterpret_cast<const uint4 *>(decision);
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    const uint4 d = __ldcs(dec4 + i);
+    one(d.x); one(d.y); one(d.z); one(d.w);
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) one(decision[(n4 << 2) + threadIdx.x]);
+  n_feas = __reduce_add_sync(0xFFFFFFFFu, n_feas);
+  n_nofeas = __reduce_add_sync(0xFFFFFFFFu, n_nofeas);
+  n_inval = __reduce_add_sync(0xFFFFFFFFu, n_inval);
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&blk[0], n_feas);
+    atomicAdd(&blk[1], n_nofeas);
+    atomicAdd(&blk[2], n_inval);
+  }
+  __syncthreads();
+  for (uint32_t i = threadIdx.x; i < n_variants; i += blockDim.x) {
+    const uint32_t h = hist[i];
+    if (h) atomicAdd(&count_by_id[i], h);
+  }
+  if (threadIdx.x < 3 && blk[threadIdx.x]) atomicAdd(&counters[threadIdx.x], (unsigned long long)blk[threadIdx.x]);
+}
+
 // ------------------------------------------------------------------------------------
 // Rebuild: one CTA per task.
 // ------------------------------------------------------------------------------------
@@ -100,75 +143,129 @@ __device__ __forceinline__ uint32_t block_excl_scan_flag(bool flag, uint32_t *wa
   return before + in_warp;
 }
 
-// Smallest slo that falls in SLO bucket b >= 1 (see common.cuh).
-__device__ __forceinline__ uint32_t slo_bucket_floor(uint32_t b) {
-  const float f = __uint_as_float((b + SLO_BUCKET_BIAS) << 20);
-  return (uint32_t)ceilf(f);     // exact: f < 2^32 and has at most 3 fractional bits
+// Top 15 bits of a u32 converted to float toward zero: a monotone, roughly logarithmic
+// code (8 exponent bits, 7 mantissa bits).  The selection kernel computes the same code.
+__device__ __forceinline__ uint32_t float_code(uint32_t x) {
+  return __float_as_uint(__uint2float_rz(x)) >> 16;
+}
+// Smallest u32 whose float_code is >= code (code > 0).
+__device__ __forceinline__ uint32_t float_code_floor(uint32_t code) {
+  return __float2uint_ru(__uint_as_float(code << 16));
 }
 
-// Builds the rank / bitmask index of a list of F <= MASK_MAX_F entries (see common.cuh).
-// fr_pred / fr_acc: the list in scan order (shared memory).  Writes into the task block.
-__device__ void build_index(unsigned char *block, const BlockLayout &L, uint32_t F,
-                            const uint32_t *fr_pred, const uint16_t *fr_acc, uint16_t *rkL,
-                            uint16_t *rkA, uint32_t *thr_s, uint16_t *acc_s, uint32_t *meta_out) {
+struct IndexScratch {          // shared memory used while building one task's index
+  uint32_t pred[256], Pd[256];
+  uint16_t acc[256], Ad[256];
+  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256];
+  uint32_t ks, ka;
+};
+
+// Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh).
+// S.pred / S.acc hold the list in scan order.  Writes the SLO records straight into the
+// image, the var block and the cold Pd array into the task's region, and the task's header
+// words (without var_base), Ks and var-block size into the per-task arrays.
+__device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint32_t V, IndexScratch &S) {
   const uint32_t tid = threadIdx.x, B = blockDim.x;
-  // ranks by counting (stable: equal values keep scan order)
+  unsigned char *region = c.regions + c.reg_off[t];
+  // distinct values and their ranks
   for (uint32_t p = tid; p < F; p += B) {
-    const uint32_t pp = fr_pred[p], pa = fr_acc[p];
-    uint32_t cl = 0, ca = 0;
-    for (uint32_t q = 0; q < F; ++q) {
-      const uint32_t qp = fr_pred[q], qa = fr_acc[q];
-      cl += (qp < pp) || (qp == pp && q < p);
-      ca += (qa < pa) || (qa == pa && q < p);
+    bool fp = true, fa = true;
+    for (uint32_t q = 0; q < p; ++q) {
+      fp &= S.pred[q] != S.pred[p];
+      fa &= S.acc[q] != S.acc[p];
     }
-    rkL[p] = (uint16_t)cl;
-    rkA[p] = (uint16_t)ca;
-    thr_s[cl] = pp;
-    acc_s[ca] = (uint16_t)pa;
+    S.firstP[p] = fp;
+    S.firstA[p] = fa;
+  }
+  if (tid == 0) { S.ks = 0; S.ka = 0; }
+  __syncthreads();
+  for (uint32_t p = tid; p < F; p += B) {
+    uint32_t rp = 0, ra = 0;
+    for (uint32_t q = 0; q < F; ++q) {
+      rp += S.firstP[q] && S.pred[q] < S.pred[p];
+      ra += S.firstA[q] && S.acc[q] < S.acc[p];
+    }
+    S.idxP[p] = (unsigned char)rp;
+    S.idxA[p] = (unsigned char)ra;
+    S.Pd[rp] = S.pred[p];
+    S.Ad[ra] = S.acc[p];
+    atomicMax(&S.ks, rp + 1);
+    atomicMax(&S.ka, ra + 1);
   }
   __syncthreads();
-  uint32_t *thr_g = reinterpret_cast<uint32_t *>(block + L.thr);
-  uint16_t *acc_g = reinterpret_cast<uint16_t *>(block + L.accs);
-  for (uint32_t i = tid; i < F; i += B) {
-    thr_g[i] = thr_s[i];
-    acc_g[i] = acc_s[i];
+  const uint32_t Ks = S.ks, Ka = S.ka;
+  // positions ordered by rank of pred_lat (ties in scan order)
+  for (uint32_t p = tid; p < F; p += B) {
+    uint32_t o = 0;
+    for (uint32_t q = 0; q < F; ++q) o += S.idxP[q] < S.idxP[p] || (S.idxP[q] == S.idxP[p] && q < p);
+    S.order[o] = (unsigned char)p;
   }
-  // bucket tables
-  const uint32_t acc_base = acc_s[0], acc_range = acc_s[F - 1] - acc_s[0];
-  uint32_t shift = 0;
-  while ((acc_range >> shift) > ACC_BUCKETS - 1) ++shift;
-  if (tid == 0) *meta_out = acc_base | (shift << 16);
-  unsigned char *startL = block + L.start, *startA = startL + SLO_BUCKET_BYTES;
-  for (uint32_t b = tid; b < SLO_BUCKET_BYTES + ACC_BUCKETS; b += B) {
-    uint32_t cnt = 0;
-    if (b < SLO_BUCKETS) {
-      if (b > 0) {
-        const uint32_t lo = slo_bucket_floor(b);       // every slo in the bucket is >= lo
-        for (uint32_t i = 0; i < F; ++i) cnt += thr_s[i] < lo;
-      }
-      startL[b] = (unsigned char)min(cnt, 255u);
-    } else if (b < SLO_BUCKET_BYTES) {
-      startL[b] = 0;
+  __syncthreads();
+  uint32_t *Pd_g = reinterpret_cast<uint32_t *>(region + 12u * V);
+  for (uint32_t i = tid; i < Ks; i += B) Pd_g[i] = S.Pd[i];
+
+  // SLO records
+  const uint32_t cmin = float_code(S.Pd[0]), cmax = float_code(S.Pd[Ks - 1]);
+  uint32_t sh = 0;
+  while ((cmax >> sh) - (cmin >> sh) > SLO_BUCKETS - 1) ++sh;
+  const uint32_t bmin = cmin >> sh;
+  uint32_t *slo_rec = reinterpret_cast<uint32_t *>(c.image + image_slo_offset(c.n_tasks)) + t * SLO_BUCKETS;
+  for (uint32_t j = tid; j < SLO_BUCKETS; j += B) {
+    uint32_t lb = 0, cnt = 0, thr = 0;
+    for (uint32_t i = 0; i < Ks; ++i) {
+      const uint32_t b = min(max(float_code(S.Pd[i]) >> sh, bmin) - bmin, SLO_BUCKETS - 1);
+      lb += b < j;
+      if (b == j) { ++cnt; thr = S.Pd[i]; }
+    }
+    uint32_t rec;
+    if (cnt == 0) {
+      rec = lb ? ((lb - 1) << 24) : 0x00FFFFFFu;   // "always one more than lb-1" / never (lb = 0)
+    } else if (cnt == 1) {
+      const uint32_t lo = j ? float_code_floor((bmin + j) << sh) : 0u;
+      const uint32_t delta = thr - lo;
+      rec = delta < 0x01000000u ? (lb << 24) | delta : (SLO_FLAGGED << 24);
     } else {
-      const uint32_t lo = acc_base + ((b - SLO_BUCKET_BYTES) << shift);   // every min_acc in the bucket is >= lo
-      for (uint32_t i = 0; i < F; ++i) cnt += acc_s[i] < lo;
-      startA[b - SLO_BUCKET_BYTES] = (unsigned char)min(cnt, 255u);
+      rec = SLO_FLAGGED << 24;
+    }
+    slo_rec[j] = rec;
+  }
+
+  // var block: ids (already written by the caller), accuracy bitmap, T2
+  const uint32_t acc_min = S.Ad[0] & ~3u;
+  const uint32_t nbw = (S.Ad[Ka - 1] - acc_min + 2u + ACC_WORD_BITS - 1u) / ACC_WORD_BITS;
+  const uint32_t Fp8 = (F + 7u) / 8u;
+  const uint32_t width = (Ka + 2u) & ~1u;                     // Ka + 1 rounded up to even
+  unsigned char *var = region + region_var_offset(V);
+  uint32_t *bitmap = reinterpret_cast<uint32_t *>(var + 32u * Fp8);
+  for (uint32_t w = tid; w < nbw; w += B) {
+    uint32_t bits = 0, prefix = 0;
+    for (uint32_t i = 0; i < Ka; ++i) {
+      const uint32_t x = S.Ad[i] - acc_min, xw = x / ACC_WORD_BITS;
+      prefix += xw < w;
+      if (xw == w) bits |= 1u << (x - xw * ACC_WORD_BITS);
+    }
+    bitmap[w] = (prefix << 24) | bits;
+  }
+  unsigned char *T2 = var + 32u * Fp8 + 4u * nbw;
+  for (uint32_t k = tid; k < width; k += B) {
+    uint32_t cur = 0xFFu, o = 0;
+    T2[k] = 0xFFu;                                             // r = 0: no latency is met
+    for (uint32_t r = 1; r <= Ks; ++r) {
+      while (o < F && S.idxP[S.order[o]] == r - 1) {
+        const uint32_t p = S.order[o];
+        if (S.idxA[p] >= k && p < cur) cur = p;
+        ++o;
+      }
+      T2[r * width + k] = (unsigned char)cur;
     }
   }
-  // masks
-  unsigned long long *ML = reinterpret_cast<unsigned long long *>(block + L.masks);
-  unsigned long long *MA = ML + (F + 1) * L.nw;
-  for (uint32_t idx = tid; idx < (F + 1) * L.nw; idx += B) {
-    const uint32_t r = idx / L.nw, w = idx - r * L.nw;
-    unsigned long long ml = 0, ma = 0;
-    const uint32_t p_end = min(F, 64u * w + 64u);
-    for (uint32_t p = 64u * w; p < p_end; ++p) {
-      const unsigned long long bit = 1ull << (p & 63u);
-      if (rkL[p] < r) ml |= bit;
-      if (rkA[p] >= r) ma |= bit;
-    }
-    ML[idx] = ml;
-    MA[idx] = ma;
+  if (tid == 0) {
+    TaskHdr h;
+    h.w0 = ((acc_min >> 2) << 12) | (sh << 24) | (Fp8 << 27);
+    h.w1 = bmin | (nbw << 15) | ((width >> 1) << 24);
+    c.f_hdr[t] = h;
+    c.f_ks[t] = Ks;
+    c.f_var_bytes[t] = round_up_u32(4u * nbw + 32u * Fp8 + (Ks + 1u) * width, 64u);
   }
 }
 
@@ -179,8 +276,7 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
   __shared__ uint32_t s_last, s_total;
-  __shared__ uint32_t fr_pred[MASK_MAX_F], thr_s[MASK_MAX_F];
-  __shared__ uint16_t fr_acc[MASK_MAX_F], rkL[MASK_MAX_F], rkA[MASK_MAX_F], acc_s[MASK_MAX_F];
+  __shared__ IndexScratch S;
 
   const uint32_t t = blockIdx.x, tid = threadIdx.x, B = blockDim.x;
   const uint32_t base = c.task_off[t];
@@ -247,8 +343,14 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   for (uint32_t p = tid; p < V; p += B) {
     const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
     bool kp = true;
-    for (uint32_t q = 0; q < p; ++q) {
-      if ((uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p) { kp = false; break; }
+    for (uint32_t q0 = 0; q0 < p && kp; q0 += 8) {     // groups of 8, exit between groups
+      bool dom = false;
+#pragma unroll
+      for (uint32_t j = 0; j < 8; ++j) {
+        const uint32_t q = min(q0 + j, p - 1);          // clamped repeats are harmless
+        dom |= (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
+      }
+      kp = !dom;
     }
     keep[p] = kp;
     my_kept += kp;
@@ -259,12 +361,13 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   if ((tid & 31) == 0 && my_kept) atomicAdd(&s_total, my_kept);
   __syncthreads();
   const uint32_t F = s_total;
-  const BlockLayout L = block_layout(F);
-  unsigned char *block = c.regions + c.reg_off[t];
+  const bool indexed = F > 0 && F <= INDEX_MAX_F;
+  unsigned char *region = c.regions + c.reg_off[t];
 
-  // 4. compact into the task block (scan order)
-  unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(block + L.keys);
-  uint32_t *ids_g = reinterpret_cast<uint32_t *>(block + L.ids);
+  // 4. compact into the task's region (scan order): cold keys and ids, and the var block's ids
+  unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(region);
+  uint32_t *ids_g = reinterpret_cast<uint32_t *>(region + 8u * V);
+  uint32_t *var_ids = reinterpret_cast<uint32_t *>(region + region_var_offset(V));
   uint32_t kept_so_far = 0;
   for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
     const uint32_t p = p0 + tid;
@@ -273,17 +376,24 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
     const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
     if (kp) {
       const uint32_t pred_p = (uint32_t)k64[p], acc = 10000u - (k32[p] >> 16);
+      const uint32_t id = c.s_id[base + (k32[p] & 0xFFFFu)];
       keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
-      ids_g[pos] = c.s_id[base + (k32[p] & 0xFFFFu)];
-      if (L.nw) { fr_pred[pos] = pred_p; fr_acc[pos] = (uint16_t)acc; }
+      ids_g[pos] = id;
+      if (indexed) { var_ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }
     }
     kept_so_far += total;
   }
   __syncthreads();
-  if (tid == 0) { c.f_len[t] = F; if (!L.nw) c.f_meta[t] = 0; }
-  if (L.nw) build_index(block, L, F, fr_pred, fr_acc, rkL, rkA, thr_s, acc_s, c.f_meta + t);
+  if (indexed) {
+    build_index(c, t, F, V, S);
+  } else if (tid == 0) {
+    c.f_hdr[t] = TaskHdr{0u, 0u};
+    c.f_ks[t] = 0;
+    c.f_var_bytes[t] = 0;
+  }
+  if (tid == 0) c.f_len[t] = F;
 
-  // 5. the CTA that finishes last packs all blocks into the image
+  // 5. the CTA that finishes last packs the var blocks into the image and writes the headers
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -295,17 +405,20 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   __threadfence();
 
   const uint32_t T = c.n_tasks;
-  TaskDesc *desc = reinterpret_cast<TaskDesc *>(c.image);
-  const uint32_t desc_bytes = T * (uint32_t)sizeof(TaskDesc);
-  // 5a. block offsets = exclusive prefix sum of block sizes (chunks of B tasks, running carry)
-  uint32_t carry = desc_bytes, longest = 0, entries = 0, linear = 0;
+  TaskHdr *hdr = reinterpret_cast<TaskHdr *>(c.image);
+  const uint32_t var0 = image_var_offset(T);
+  // 5a. var offsets = exclusive prefix sum of the var-block sizes (chunks of B tasks)
+  uint32_t carry = 0, longest = 0, entries = 0, not_indexed = 0;
   __shared__ uint32_t scan_buf[1024];
-  bool overflow = false;
+  __shared__ uint32_t s_copy_end;
+  bool overflow = var0 > c.image_capacity;
   for (uint32_t t0 = 0; t0 < T; t0 += B) {
     const uint32_t tt = t0 + tid;
     const uint32_t len = tt < T ? __ldcg(c.f_len + tt) : 0u;
-    const BlockLayout Lt = block_layout(len);
-    scan_buf[tid] = Lt.bytes;
+    uint32_t vbytes = tt < T ? __ldcg(c.f_var_bytes + tt) : 0u;
+    // a block that would start beyond what var_base can address is left out: the task is
+    // then served by the slow path (decided per task below, after the scan)
+    scan_buf[tid] = vbytes;
     __syncthreads();
     for (uint32_t o = 1; o < B; o <<= 1) {      // Hillis-Steele inclusive scan
       uint32_t v = tid >= o ? scan_buf[tid - o] : 0u;
@@ -316,52 +429,78 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
     const uint32_t chunk_total = scan_buf[B - 1];
     const uint32_t incl = scan_buf[tid];
     __syncthreads();                                               // scan_buf is reused below
-    if (carry + chunk_total > c.image_capacity) overflow = true;   // uniform
+    if (var0 + carry + chunk_total > c.image_capacity) overflow = true;   // uniform
+    const uint32_t off = carry + incl - vbytes;                    // from the start of the var section
+    const bool addressable = (off >> 6) < VB_NOT_INDEXED;
     if (tt < T && !overflow) {
-      const uint32_t off = carry + incl - Lt.bytes;
-      TaskDesc d;
-      d.off_masks = off + Lt.masks;
-      d.f_nw = len | (Lt.nw << 16);
-      d.acc_meta = __ldcg(c.f_meta + tt);
-      d.off_keys = off + Lt.keys;
-      d.off_thr = off + Lt.thr;
-      d.off_ids = off + Lt.ids;
-      d.off_accs = off + Lt.accs;
-      d.off_start = off + Lt.start;
-      desc[tt] = d;
-      // the block's offset, kept for the copy pass
-      scan_buf[tid] = off;
+      const uint2 raw = __ldcg(reinterpret_cast<const uint2 *>(c.f_hdr + tt));
+      TaskHdr h{raw.x, raw.y};
+      uint32_t vb;
+      if (len == 0) vb = VB_NO_VARIANTS;
+      else if (vbytes == 0 || !addressable) vb = VB_NOT_INDEXED;
+      else vb = off >> 6;
+      h.w0 = (h.w0 & ~0xFFFu) | vb;
+      hdr[tt] = h;
+      not_indexed += (vb == VB_NOT_INDEXED);
     }
+    // offsets stay ascending: empty blocks share the next block's offset, and the blocks
+    // that are left out (and the padding past T) form a suffix of sentinels
+    scan_buf[tid] = (tt < T && addressable) ? off : 0xFFFFFFFFu;
+    if (tid == 0) s_copy_end = carry;
     __syncthreads();
-    // 5b. copy this chunk's blocks (one warp per task, 16 bytes per lane and step)
+    if (tt < T && addressable && vbytes) atomicMax(&s_copy_end, off + vbytes);
+    __syncthreads();
+    // 5b. copy this chunk's var blocks: 16-byte units spread over all threads; a unit finds
+    // its block by binary search over the chunk's ascending offsets
     if (!overflow) {
-      const uint32_t lane = tid & 31, warp = tid >> 5, nwarps = B >> 5;
-      for (uint32_t i = warp; i < B && t0 + i < T; i += nwarps) {
-        const uint32_t len_i = __ldcg(c.f_len + t0 + i);
-        const uint32_t bytes_i = block_layout(len_i).bytes;
-        const uint4 *src = reinterpret_cast<const uint4 *>(c.regions + c.reg_off[t0 + i]);
-        uint4 *dst = reinterpret_cast<uint4 *>(c.image + scan_buf[i]);
-        for (uint32_t e = lane; e < (bytes_i >> 4); e += 32) dst[e] = __ldcg(src + e);
+      const uint32_t units = (s_copy_end - carry) >> 4;
+      const uint4 *reg4 = reinterpret_cast<const uint4 *>(c.regions);
+      uint4 *img4 = reinterpret_cast<uint4 *>(c.image + var0);
+      for (uint32_t u0 = 0; u0 < units; u0 += 4u * B) {
+        uint4 v[4];
+        uint32_t dst[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t u = u0 + (uint32_t)j * B + tid;
+          dst[j] = 0xFFFFFFFFu;
+          if (u < units) {
+            const uint32_t byte = carry + (u << 4);
+            uint32_t lo = 0, hi = B;                    // last i with scan_buf[i] <= byte
+            while (hi - lo > 1) {
+              const uint32_t mid = (lo + hi) >> 1;
+              if (scan_buf[mid] <= byte) lo = mid; else hi = mid;
+            }
+            {
+              const uint32_t tsrc = t0 + lo;
+              const uint32_t Vt = __ldg(c.task_off + tsrc + 1) - __ldg(c.task_off + tsrc);
+              const uint32_t src_byte = __ldg(c.reg_off + tsrc) + region_var_offset(Vt) + (byte - scan_buf[lo]);
+              v[j] = __ldcg(reg4 + (src_byte >> 4));
+              dst[j] = byte >> 4;
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (dst[j] != 0xFFFFFFFFu) img4[dst[j]] = v[j];
       }
     }
     longest = max(longest, len);
     entries += len;
-    linear += (len > 0 && Lt.nw == 0);
     __syncthreads();
     carry += chunk_total;
   }
   // totals for reporting
   longest = __reduce_max_sync(0xFFFFFFFFu, longest);
   entries = __reduce_add_sync(0xFFFFFFFFu, entries);
-  linear = __reduce_add_sync(0xFFFFFFFFu, linear);
+  not_indexed = __reduce_add_sync(0xFFFFFFFFu, not_indexed);
   __shared__ uint32_t tot[3];
   if (tid == 0) tot[0] = tot[1] = tot[2] = 0;
   __syncthreads();
-  if ((tid & 31) == 0) { atomicMax(&tot[0], longest); atomicAdd(&tot[1], entries); atomicAdd(&tot[2], linear); }
+  if ((tid & 31) == 0) { atomicMax(&tot[0], longest); atomicAdd(&tot[1], entries); atomicAdd(&tot[2], not_indexed); }
   __syncthreads();
   if (tid == 0) {
     if (overflow) atomicMax(c.err, (uint32_t)DEV_ERR_IMAGE_OVERFLOW);
-    c.image_hdr[0] = overflow ? 0xFFFFFFFFu : carry;
+    c.image_hdr[0] = overflow ? 0xFFFFFFFFu : var0 + carry;
     c.image_hdr[1] = tot[0];
     c.image_hdr[2] = tot[1];
     c.image_hdr[3] = tot[2];
@@ -371,9 +510,23 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
 
 }  // namespace
 
+constexpr uint32_t TALLY_SMEM_MAX_VARIANTS = 49152;   // 192 KB of bins
+constexpr uint64_t TALLY_SMEM_MIN_N = 1u << 18;        // below this the zero/flush passes cost more than they save
+
 cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uint64_t n,
                          cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
+  if (n >= TALLY_SMEM_MIN_N && c.n_variants <= TALLY_SMEM_MAX_VARIANTS) {
+    const size_t smem = (size_t)c.n_variants * 4;
+    const uint32_t per_sm = smem > 100 * 1024 ? 1 : 2;
+    uint64_t want = ((n >> 2) + TALLY_SMEM_THREADS * 8 - 1) / (TALLY_SMEM_THREADS * 8);
+    uint64_t grid = (uint64_t)148 * per_sm;
+    if (grid > want) grid = want;
+    if (grid < 1) grid = 1;
+    tally_smem_kernel<<<(uint32_t)grid, TALLY_SMEM_THREADS, smem, stream>>>(
+        d_decision, n, c.n_variants, c.count_by_id, c.counters);
+    return cudaGetLastError();
+  }
   uint64_t want = ((n >> 2) + 255) / 256;
   uint32_t grid = (uint32_t)(want < 1 ? 1 : (want > 148 * 8 ? 148 * 8 : want));
   tally_kernel<<<grid, 256, 0, stream>>>(d_decision, n, c.n_variants, c.count_by_id, c.counters);
@@ -381,6 +534,9 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
 }
 
 cudaError_t prepare_rebuild_kernel() {
+  cudaError_t e = cudaFuncSetAttribute(tally_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)(TALLY_SMEM_MAX_VARIANTS * 4));
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(rebuild_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)REBUILD_MAX_SMEM);
 }
@@ -389,7 +545,7 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream) {
   uint32_t P = 1;
   while (P < c.max_task_variants) P <<= 1;
-  uint32_t block = P < 128 ? 128 : (P > 1024 ? 1024 : P);
+  uint32_t block = P < 256 ? 256 : (P > 1024 ? 1024 : P);
   size_t smem = (size_t)P * 13;
   rebuild_kernel<<<c.n_tasks, block, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
   return cudaGetLastError();
