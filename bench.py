@@ -264,6 +264,7 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
     value = world * n / (ms_per_step * 1e-3)
     state = P.infaas_catalog_get_state(cat)
+    info = P.infaas_catalog_get_info(cat)
     dec_host = d_dec.cpu().numpy().view(np.uint32)
 
     peak, peak_kind = measured_hbm_peak()
@@ -288,6 +289,7 @@ def run_ours(args):
                       "no_feasible": int((((dec_host >> 31) == 1) & (dec_host != 0xFFFFFFFF)).sum()),
                       "invalid": int((dec_host == 0xFFFFFFFF).sum()),
                       "queued_max": int(state["queued"].max())},
+        "lookup": dict(info, staged_in_shared_memory=info["image_bytes"] <= info["image_smem"]),
     }
 
     if not args.no_extras:

@@ -134,6 +134,16 @@ int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_
 int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_ids,
                                 uint32_t cap, uint32_t *h_len, void *cuda_stream);
 
+/* Sizes of the structures built for the current load state, for reporting (HOST array):
+ *   h_info[0] bytes of the packed lookup image the selection kernel reads
+ *   h_info[1] longest per-task scan list        h_info[2] sum of the list lengths
+ *   h_info[3] tasks whose list has no rank index (longer than the index supports)
+ *   h_info[4] shared memory (bytes) the next infaas_select_batch reserves for the image;
+ *             if h_info[0] is larger the kernel reads the image from global memory
+ *   h_info[5..7] reserved (0).
+ * Synchronises cuda_stream. */
+int infaas_catalog_get_info(infaas_catalog *c, uint32_t h_info[8], void *cuda_stream);
+
 /* (No counterpart in the paper: an addition for callers that cannot allocate.)
  * Per-variant tallies of a decision array, as the first step of infaas_load_update computes
  * them, for callers that must not trigger a device allocation: a serving process that has

@@ -21,7 +21,7 @@ _lib = None
 
 EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
-           "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static")
+           "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info")
 
 
 class InfaasError(RuntimeError):
@@ -47,6 +47,8 @@ def _load():
     lib.infaas_load_update.argtypes = [vp, vp, u64, u32, vp]
     lib.infaas_catalog_get_state.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.infaas_catalog_get_frontier.argtypes = [vp, u32, vp, u32, ctypes.POINTER(u32), vp]
+    lib.infaas_catalog_get_info.argtypes = [vp, vp, vp]
+    lib.infaas_catalog_get_info.restype = i32
     lib.infaas_catalog_free.argtypes = [vp]
     lib.infaas_catalog_free.restype = None
     for name in ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
@@ -140,6 +142,14 @@ def infaas_catalog_get_state(cat: Catalog, stream=None) -> dict:
     return {"queued": queued, "pred_lat_us": pred, "served_total": served, "counters": counters}
 
 
+def infaas_catalog_get_info(cat: Catalog, stream=None) -> dict:
+    info = np.zeros(8, np.uint32)
+    _check(_load().infaas_catalog_get_info(cat.handle, info.ctypes.data, _stream_ptr(stream)),
+           "infaas_catalog_get_info")
+    return {"image_bytes": int(info[0]), "longest_list": int(info[1]), "list_entries": int(info[2]),
+            "tasks_not_indexed": int(info[3]), "image_smem": int(info[4])}
+
+
 def infaas_catalog_get_frontier(cat: Catalog, task: int, stream=None) -> np.ndarray:
     ids = np.empty(max(1, cat.n_variants), np.uint32)
     ln = ctypes.c_uint32(0)
@@ -161,4 +171,4 @@ def infaas_tally_static(d_decision, n_variants: int, d_count, d_counters, n=None
         raise ValueError("d_count is shorter than n_variants")
     _check(_load().infaas_tally_static(_dev_ptr(d_decision, "u32"), n, int(n_variants),
                                        _dev_ptr(d_count, "u32"), d_counters.data_ptr(),
-                                       d_count.device.index, _stream_ptr(stream)), "infaas_tally_static")
+                                       d_count.device.index, _stream_ptr(stream)), "infaas_tally_static", "infaas_catalog_get_info")

@@ -319,6 +319,20 @@ int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_id
   return INFAAS_OK;
 }
 
+int infaas_catalog_get_info(infaas_catalog *c, uint32_t h_info[8], void *cuda_stream) {
+  if (!c || !h_info) return INFAAS_E_NULL;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t hdr[4] = {0, 0, 0, 0};
+  CUDA_TRY(cudaMemcpyAsync(hdr, c->d.image_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  for (int i = 0; i < 4; ++i) h_info[i] = hdr[i];
+  h_info[4] = infaas::select_image_smem(c->select_smem);
+  h_info[5] = h_info[6] = h_info[7] = 0;
+  return INFAAS_OK;
+}
+
 void infaas_catalog_free(infaas_catalog *c) {
   if (!c) return;
   if (c->arena) {

@@ -22,20 +22,26 @@ namespace infaas {
 // r comes from a table of SLO_BUCKETS records indexed by a monotone bucket of slo (top bits
 // of slo converted to float, shifted by `sh`, relative to `bmin`); a record holds the rank
 // below the bucket and the one distinct value inside it (as a 24-bit offset from the
-// bucket's smallest slo); buckets with two or more values are flagged and such queries take
-// the exact slow path.  k comes from a bitmap over acc values with running popcounts (24
-// bitmap bits + 8 prefix bits per word), exact at one basis point.
+// bucket's smallest slo); a bucket with two or more values is flagged and its record gives
+// the range of Pd to compare against instead.  k comes from a bitmap over acc values with
+// running popcounts (24 bitmap bits + 8 prefix bits per word), exact at one basis point.
 //
 // Image (what the selection kernel stages in shared memory), all parts 64-byte aligned:
 //   hdr   u64[n_tasks]            per-task packed parameters (TaskHdr below)
-//   slo   u32[n_tasks][SLO_BUCKETS]   SLO records: lb << 24 | delta ; lb == 0xFF: flagged
-//   var   per-task blocks back to back, each: ids u32[8*Fp8], acc bitmap u32[nbw],
-//         T2 u8[(Ks+1)*width], padded to 64 bytes
+//   slo   u32[n_tasks][SLO_BUCKETS]   SLO records: lb << 24 | delta, or flagged:
+//                                     0xFF << 24 | lb << 8 | number of values in the bucket
+//   var   per-task blocks back to back, each: ids u32[8*Fp8], Pd u32[8*Fp8],
+//         acc bitmap u32[nbw], T2 u8[(Ks+1)*width], padded to 64 bytes
 //
 // Cold data (read from global memory by the slow path only), per task in its region, V =
 // number of the task's variants:
 //   keys u64[V] (F used)  pred_lat | acc_bp << 32 in scan order;  ids u32[V] (F used);
-//   Pd u32[Ks];  then, 64-byte aligned, the var block before it is packed into the image
+//   then, for an indexed list (Fi = min(V, INDEX_MAX_F)), what the nearest-miss search uses:
+//   bestA u8[Fi+1]   bestA[r]: position of the highest accuracy among the r smallest latencies
+//   bestB u8[Fi+1]   bestB[k]: position of the lowest latency among all but the k smallest accuracies
+//   order u8[Fi]     positions sorted by latency rank;  ordStart u8[Fi+1]: first index of rank r
+//   idxA u8[Fi], idxP u8[Fi]   accuracy / latency rank of each position
+//   then, 64-byte aligned, the var block before it is packed into the image
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
@@ -62,12 +68,26 @@ inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) {
 // Worst-case bytes of one task's var block and of its region (cold data + var block).
 inline __host__ __device__ uint32_t var_capacity(uint32_t V) {
   const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
-  return round_up_u32(4u * MAX_ACC_WORDS + 4u * round_up_u32(F, 8) + (F + 1u) * (F + 2u), 64u);
+  return round_up_u32(4u * MAX_ACC_WORDS + 8u * round_up_u32(F, 8) + (F + 1u) * (F + 2u), 64u);
 }
-inline __host__ __device__ uint32_t region_var_offset(uint32_t V) {
-  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
-  return round_up_u32(12u * V + 4u * F, 64u);     // after keys[V], ids[V] and Pd[min(V, INDEX_MAX_F)]
+struct ColdLayout {    // byte offsets inside a task's region
+  uint32_t keys, ids, bestA, bestB, order, ordStart, idxA, idxP, var;
+};
+inline __host__ __device__ ColdLayout cold_layout(uint32_t V) {
+  const uint32_t Fi = V < INDEX_MAX_F ? V : INDEX_MAX_F;
+  ColdLayout L;
+  L.keys = 0;
+  L.ids = 8u * V;
+  L.bestA = 12u * V;
+  L.bestB = L.bestA + Fi + 1u;
+  L.order = L.bestB + Fi + 1u;
+  L.ordStart = L.order + Fi;
+  L.idxA = L.ordStart + Fi + 1u;
+  L.idxP = L.idxA + Fi;
+  L.var = round_up_u32(L.idxP + Fi, 64u);
+  return L;
 }
+inline __host__ __device__ uint32_t region_var_offset(uint32_t V) { return cold_layout(V).var; }
 inline __host__ __device__ uint32_t region_capacity(uint32_t V) {
   return region_var_offset(V) + var_capacity(V);
 }
@@ -95,7 +115,7 @@ struct DeviceCatalog {
 
   unsigned char *regions;    // per task: keys, Pd, then the var block before packing
   uint32_t *f_len;           // [n_tasks] list length F
-  uint32_t *f_ks;            // [n_tasks] number of distinct pred_lat values (0 if not indexed)
+  uint32_t *f_ks;            // [n_tasks] Ks | Ka << 16: distinct pred_lat / acc_bp values (0 if not indexed)
   uint32_t *f_var_bytes;     // [n_tasks] bytes of the task's var block (0 if not indexed)
   TaskHdr *f_hdr;            // [n_tasks] header words without var_base (filled in when packing)
 
@@ -133,6 +153,8 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
 // `image_smem`: bytes of dynamic shared memory reserved for the staged image (multiple of
 // 16).  If the image is larger at run time the kernel reads it from global memory instead.
 // Returns cudaErrorInvalidValue if n is too large for the launch geometry.
+// Shared memory the launcher actually reserves for the image when asked for `image_smem`.
+uint32_t select_image_smem(uint32_t image_smem);
 cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const uint32_t *d_slo,
                           const uint16_t *d_min_acc, uint64_t n, uint32_t *d_decision,
                           int sm_count, uint32_t image_smem, cudaStream_t stream);

@@ -12,9 +12,9 @@
 // common.cuh): five shared-memory loads per query, no loop.  The packed image of all
 // tasks is staged in shared memory once per CTA with bulk asynchronous copies (TMA,
 // mbarrier completion); queries stream through with 128-bit loads and stores, four per
-// thread and iteration.  Queries that need more (no feasible variant, a flagged SLO bucket,
-// a task whose list is too long for the index) are parked in a per-warp list and resolved
-// exactly 32 at a time with all lanes busy.
+// thread and iteration.  Queries without a feasible variant (and those of a task whose list
+// is too long for the index) are parked in a per-warp list and resolved 32 at a time with
+// all lanes busy.
 #include "common.cuh"
 
 namespace infaas {
@@ -96,7 +96,7 @@ struct GlobalImage {
 
 // Per-task parameters unpacked from the two header words (see common.cuh).
 struct TaskParams {
-  uint32_t vb, acc_min, sh, ids_off, bitmap_off, t2_off, bmin, nbw, width;
+  uint32_t vb, acc_min, sh, ids_off, pd_off, bitmap_off, t2_off, bmin, nbw, width;
 };
 __device__ __forceinline__ TaskParams unpack_hdr(uint32_t w0, uint32_t w1, uint32_t var0) {
   TaskParams P;
@@ -107,9 +107,28 @@ __device__ __forceinline__ TaskParams unpack_hdr(uint32_t w0, uint32_t w1, uint3
   P.nbw = (w1 >> 15) & 0x1FFu;
   P.width = ((w1 >> 24) & 0x7Fu) << 1;
   P.ids_off = var0 + (P.vb << 6);
-  P.bitmap_off = P.ids_off + ((w0 >> 27) << 5);
+  P.pd_off = P.ids_off + ((w0 >> 27) << 5);
+  P.bitmap_off = P.pd_off + ((w0 >> 27) << 5);
   P.t2_off = P.bitmap_off + (P.nbw << 2);
   return P;
+}
+
+// r = #{distinct list latencies <= slo}: one bucket record and one comparison; a flagged
+// bucket (two or more values inside) compares against that short range of Pd instead.
+template <class Img>
+__device__ __forceinline__ uint32_t slo_rank(const Img &img, const TaskParams &P, uint32_t slo_off,
+                                             uint32_t task, uint32_t slo) {
+  const uint32_t b = (__float_as_uint(__uint2float_rz(slo)) >> 16) >> P.sh;
+  const uint32_t j = min(max(b, P.bmin) - P.bmin, SLO_BUCKETS - 1u);
+  const uint32_t lo = j ? __float2uint_ru(__uint_as_float(((P.bmin + j) << P.sh) << 16)) : 0u;
+  const uint32_t rec = img.u32(slo_off + ((task * SLO_BUCKETS + j) << 2));
+  uint32_t r = (rec >> 24) + ((slo - lo) >= (rec & 0x00FFFFFFu));
+  if ((rec >> 24) == SLO_FLAGGED) {
+    r = (rec >> 8) & 0xFFFFu;
+    const uint32_t end = r + (rec & 0xFFu);
+    for (uint32_t i = r; i < end; ++i) r += img.u32(P.pd_off + (i << 2)) <= slo;
+  }
+  return r;
 }
 
 // k = #{distinct list accuracies < min_acc}, from the bitmap with running popcounts.
@@ -121,8 +140,8 @@ __device__ __forceinline__ uint32_t acc_rank(const Img &img, const TaskParams &P
   return (word >> 24) + __popc(word & ((1u << (x - w * ACC_WORD_BITS)) - 1u));
 }
 
-// Fast path, no loops: the decision, INFAAS_INVALID, or PENDING when the query has to take
-// the exact slow path (flagged SLO bucket, task without index) or nothing is feasible.
+// Fast path: the decision, INFAAS_INVALID, or PENDING when nothing is feasible or the
+// task's list has no index (the parked query is then resolved by decide_slow).
 template <class Img>
 __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks, uint32_t slo_off,
                                                 uint32_t var0, uint32_t task, uint32_t slo,
@@ -131,56 +150,80 @@ __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks
   const uint2 h = img.v2(task << 3);
   const TaskParams P = unpack_hdr(h.x, h.y, var0);
   if (P.vb >= VB_NOT_INDEXED) return P.vb == VB_NO_VARIANTS ? INFAAS_INVALID : PENDING;
-  // r = #{distinct list latencies <= slo}: bucket record + one comparison
-  const uint32_t b = (__float_as_uint(__uint2float_rz(slo)) >> 16) >> P.sh;
-  const uint32_t j = min(max(b, P.bmin) - P.bmin, SLO_BUCKETS - 1u);
-  const uint32_t lo = j ? __float2uint_ru(__uint_as_float(((P.bmin + j) << P.sh) << 16)) : 0u;
-  const uint32_t rec = img.u32(slo_off + ((task * SLO_BUCKETS + j) << 2));
-  const uint32_t lb = rec >> 24;
-  const uint32_t r = lb == SLO_FLAGGED ? 0u : lb + ((slo - lo) >= (rec & 0x00FFFFFFu));
+  const uint32_t r = slo_rank(img, P, slo_off, task, slo);
   const uint32_t k = acc_rank(img, P, min_acc);
   const uint32_t pos = img.u8(P.t2_off + r * P.width + k);
-  if (lb == SLO_FLAGGED || pos == 0xFFu) return PENDING;
+  if (pos == 0xFFu) return PENDING;
   return img.u32(P.ids_off + (pos << 2));
 }
 
-// Exact slow path for a parked query: the decision, or the nearest miss when nothing is
-// feasible: d = 10^4 * over_lat + slo * under_acc (64-bit); strict '<' keeps the first of
-// equal distances, i.e. the smallest (cost, pred_lat, -acc, id).  Cold data comes from the
-// task's region in global memory.
+// d = 10^4 * over_lat + slo * under_acc of one list entry (64-bit).
+__device__ __forceinline__ unsigned long long miss_distance(unsigned long long key, uint32_t slo,
+                                                            uint32_t min_acc) {
+  const uint32_t pred = (uint32_t)key, acc = (uint32_t)(key >> 32);
+  const uint32_t over = pred > slo ? pred - slo : 0u;
+  const uint32_t under = min_acc > acc ? min_acc - acc : 0u;
+  return (unsigned long long)over * 10000ull + (unsigned long long)slo * under;
+}
+
+// Slow path for a parked query.  The nearest miss is the entry smallest in (d, position):
+// position order is (cost, pred_lat, -acc, id) order.  Cold data comes from the task's
+// region in global memory.
+//   Indexed list: nothing is feasible (the fast path said so).  Entries that meet the SLO
+//   all miss the accuracy, and the best of them is the one with the highest accuracy
+//   (bestA); entries that meet the accuracy all miss the SLO, the best being the one with
+//   the lowest latency (bestB); an entry that misses both can only win if its accuracy is
+//   above bestA's and its latency not above bestB's, so only that rank rectangle is walked.
+//   List without index: walk it, first for a feasible entry, then for the distance.
 template <class Img>
-__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t var0,
-                                                uint32_t task, uint32_t slo, uint32_t min_acc) {
-  const uint32_t F = __ldg(c.f_len + task), Ks = __ldg(c.f_ks + task);
+__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t slo_off,
+                                                uint32_t var0, uint32_t task, uint32_t slo,
+                                                uint32_t min_acc) {
+  const uint32_t F = __ldg(c.f_len + task);
   const uint32_t V = __ldg(c.task_off + task + 1) - __ldg(c.task_off + task);
   const unsigned char *region = c.regions + __ldg(c.reg_off + task);
+  const ColdLayout CL = cold_layout(V);
   const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(region);
-  const uint32_t *ids = reinterpret_cast<const uint32_t *>(region + 8u * V);
+  const uint32_t *ids = reinterpret_cast<const uint32_t *>(region + CL.ids);
   const uint2 h = img.v2(task << 3);
   const TaskParams P = unpack_hdr(h.x, h.y, var0);
-  if (P.vb < VB_NOT_INDEXED) {
-    const uint32_t *Pd = reinterpret_cast<const uint32_t *>(region + 12u * V);
-    uint32_t lo = 0, hi = Ks;                          // r = #{Pd <= slo}
-    while (lo < hi) {
-      const uint32_t mid = (lo + hi) >> 1;
-      if (__ldg(Pd + mid) <= slo) lo = mid + 1; else hi = mid;
-    }
-    const uint32_t pos = img.u8(P.t2_off + lo * P.width + acc_rank(img, P, min_acc));
-    if (pos != 0xFFu) return __ldg(ids + pos);
-  } else {
-    for (uint32_t i = 0; i < F; ++i) {
-      const unsigned long long e = __ldg(keys + i);
-      if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return __ldg(ids + i);
-    }
-  }
   unsigned long long best = ~0ull;
   uint32_t best_i = 0;
+  if (P.vb < VB_NOT_INDEXED) {
+    const uint32_t kk = __ldg(c.f_ks + task), Ks = kk & 0xFFFFu, Ka = kk >> 16;
+    const uint32_t r = slo_rank(img, P, slo_off, task, slo);
+    const uint32_t k = acc_rank(img, P, min_acc);
+    uint32_t acc_rank_floor = 0;          // candidates need accuracy rank >= this
+    uint32_t lat_rank_cap = Ks;           // ... and latency rank < this
+    if (r > 0) {                          // some entry meets the SLO
+      const uint32_t pA = __ldg(region + CL.bestA + r);
+      best = miss_distance(__ldg(keys + pA), slo, min_acc);
+      best_i = pA;
+      acc_rank_floor = __ldg(region + CL.idxA + pA) + 1u;
+    }
+    if (k < Ka) {                         // some entry meets the accuracy
+      const uint32_t pB = __ldg(region + CL.bestB + k);
+      const unsigned long long d = miss_distance(__ldg(keys + pB), slo, min_acc);
+      if (d < best || (d == best && pB < best_i)) { best = d; best_i = pB; }
+      lat_rank_cap = __ldg(region + CL.idxP + pB) + 1u;
+    }
+    for (uint32_t o = __ldg(region + CL.ordStart + r); o < F; ++o) {   // latency ranks >= r
+      const uint32_t p = __ldg(region + CL.order + o);
+      if (__ldg(region + CL.idxP + p) >= lat_rank_cap) break;
+      const uint32_t ia = __ldg(region + CL.idxA + p);
+      if (ia >= acc_rank_floor && ia < k) {
+        const unsigned long long d = miss_distance(__ldg(keys + p), slo, min_acc);
+        if (d < best || (d == best && p < best_i)) { best = d; best_i = p; }
+      }
+    }
+    return INFAAS_NO_FEASIBLE | __ldg(ids + best_i);
+  }
   for (uint32_t i = 0; i < F; ++i) {
     const unsigned long long e = __ldg(keys + i);
-    const uint32_t pred = (uint32_t)e, acc = (uint32_t)(e >> 32);
-    const uint32_t over = pred > slo ? pred - slo : 0u;
-    const uint32_t under = min_acc > acc ? min_acc - acc : 0u;
-    const unsigned long long d = (unsigned long long)over * 10000ull + (unsigned long long)slo * under;
+    if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return __ldg(ids + i);
+  }
+  for (uint32_t i = 0; i < F; ++i) {
+    const unsigned long long d = miss_distance(__ldg(keys + i), slo, min_acc);
     if (d < best) { best = d; best_i = i; }
   }
   return INFAAS_NO_FEASIBLE | __ldg(ids + best_i);
@@ -195,13 +238,13 @@ struct Queries {
 
 // Resolve up to 32 parked queries, one per lane.  `rel` is the query's offset from `q0`.
 template <class Img>
-__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, uint32_t var0,
-                                               const Queries &q, uint64_t q0, const uint32_t *park,
+__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, uint32_t slo_off,
+                                               uint32_t var0, const Queries &q, uint64_t q0, const uint32_t *park,
                                                uint32_t first, uint32_t count) {
   const uint32_t lane = threadIdx.x & 31;
   if (lane < count) {
     const uint64_t i = q0 + park[first + lane];
-    q.decision[i] = decide_slow(img, c, var0, q.task[i], q.slo[i], q.min_acc[i]);
+    q.decision[i] = decide_slow(img, c, slo_off, var0, q.task[i], q.slo[i], q.min_acc[i]);
   }
 }
 
@@ -270,7 +313,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
       __syncwarp();
       while (parked >= 32) {
         parked -= 32;
-        resolve_parked(img, c, var0, q, q0, park, parked, 32);
+        resolve_parked(img, c, slo_off, var0, q, q0, park, parked, 32);
       }
       __syncwarp();
     }
@@ -291,11 +334,11 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
     __syncwarp();
     while (parked >= 32) {
       parked -= 32;
-      resolve_parked(img, c, var0, q, q0, park, parked, 32);
+      resolve_parked(img, c, slo_off, var0, q, q0, park, parked, 32);
     }
   }
   __syncwarp();
-  resolve_parked(img, c, var0, q, q0, park, 0, parked);
+  resolve_parked(img, c, slo_off, var0, q, q0, park, 0, parked);
 }
 
 __global__ void __launch_bounds__(SELECT_THREADS, 1)
@@ -326,11 +369,16 @@ cudaError_t prepare_select_kernel() {
                               (int)SELECT_MAX_SMEM);
 }
 
+uint32_t select_image_smem(uint32_t image_smem) {
+  if (image_smem + PARK_BYTES > SELECT_MAX_SMEM) image_smem = (SELECT_MAX_SMEM - PARK_BYTES) & ~15u;
+  return image_smem;
+}
+
 cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const uint32_t *d_slo,
                           const uint16_t *d_min_acc, uint64_t n, uint32_t *d_decision,
                           int sm_count, uint32_t image_smem, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
-  if (image_smem + PARK_BYTES > SELECT_MAX_SMEM) image_smem = (SELECT_MAX_SMEM - PARK_BYTES) & ~15u;
+  image_smem = select_image_smem(image_smem);
   // one CTA per SM; every CTA takes one contiguous range, a multiple of the warp tile
   uint64_t grid = (uint64_t)sm_count;
   const uint64_t tiles = (n + WARP_TILE - 1) / WARP_TILE;

@@ -201,8 +201,35 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     S.order[o] = (unsigned char)p;
   }
   __syncthreads();
-  uint32_t *Pd_g = reinterpret_cast<uint32_t *>(region + 12u * V);
-  for (uint32_t i = tid; i < Ks; i += B) Pd_g[i] = S.Pd[i];
+  const ColdLayout CL = cold_layout(V);
+  const uint32_t Fp8 = (F + 7u) / 8u;
+  unsigned char *var = region + CL.var;
+  uint32_t *Pd_hot = reinterpret_cast<uint32_t *>(var + 32u * Fp8);
+  for (uint32_t i = tid; i < Ks; i += B) Pd_hot[i] = S.Pd[i];
+  // what the nearest-miss search reads (cold)
+  for (uint32_t p = tid; p < F; p += B) {
+    region[CL.order + p] = S.order[p];
+    region[CL.idxA + p] = S.idxA[p];
+    region[CL.idxP + p] = S.idxP[p];
+  }
+  for (uint32_t r = tid; r <= Ks; r += B) {
+    uint32_t best = 0xFFu, best_acc = 0, cnt = 0;           // highest accuracy among ranks < r
+    for (uint32_t p = 0; p < F; ++p) {
+      if (S.idxP[p] < r) {
+        ++cnt;
+        if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
+      }
+    }
+    region[CL.bestA + r] = (unsigned char)best;
+    region[CL.ordStart + r] = (unsigned char)cnt;
+  }
+  for (uint32_t k = tid; k <= Ka; k += B) {
+    uint32_t best = 0xFFu, best_pred = 0;                    // lowest latency among accuracy ranks >= k
+    for (uint32_t p = 0; p < F; ++p) {
+      if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
+    }
+    region[CL.bestB + k] = (unsigned char)best;
+  }
 
   // SLO records
   const uint32_t cmin = float_code(S.Pd[0]), cmax = float_code(S.Pd[Ks - 1]);
@@ -223,20 +250,18 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     } else if (cnt == 1) {
       const uint32_t lo = j ? float_code_floor((bmin + j) << sh) : 0u;
       const uint32_t delta = thr - lo;
-      rec = delta < 0x01000000u ? (lb << 24) | delta : (SLO_FLAGGED << 24);
+      rec = delta < 0x01000000u ? (lb << 24) | delta : (SLO_FLAGGED << 24) | (lb << 8) | 1u;
     } else {
-      rec = SLO_FLAGGED << 24;
+      rec = (SLO_FLAGGED << 24) | (lb << 8) | cnt;
     }
     slo_rec[j] = rec;
   }
 
-  // var block: ids (already written by the caller), accuracy bitmap, T2
+  // var block: ids (already written by the caller), Pd (above), accuracy bitmap, T2
   const uint32_t acc_min = S.Ad[0] & ~3u;
   const uint32_t nbw = (S.Ad[Ka - 1] - acc_min + 2u + ACC_WORD_BITS - 1u) / ACC_WORD_BITS;
-  const uint32_t Fp8 = (F + 7u) / 8u;
   const uint32_t width = (Ka + 2u) & ~1u;                     // Ka + 1 rounded up to even
-  unsigned char *var = region + region_var_offset(V);
-  uint32_t *bitmap = reinterpret_cast<uint32_t *>(var + 32u * Fp8);
+  uint32_t *bitmap = reinterpret_cast<uint32_t *>(var + 64u * Fp8);
   for (uint32_t w = tid; w < nbw; w += B) {
     uint32_t bits = 0, prefix = 0;
     for (uint32_t i = 0; i < Ka; ++i) {
@@ -246,7 +271,7 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     }
     bitmap[w] = (prefix << 24) | bits;
   }
-  unsigned char *T2 = var + 32u * Fp8 + 4u * nbw;
+  unsigned char *T2 = var + 64u * Fp8 + 4u * nbw;
   for (uint32_t k = tid; k < width; k += B) {
     uint32_t cur = 0xFFu, o = 0;
     T2[k] = 0xFFu;                                             // r = 0: no latency is met
@@ -264,8 +289,8 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     h.w0 = ((acc_min >> 2) << 12) | (sh << 24) | (Fp8 << 27);
     h.w1 = bmin | (nbw << 15) | ((width >> 1) << 24);
     c.f_hdr[t] = h;
-    c.f_ks[t] = Ks;
-    c.f_var_bytes[t] = round_up_u32(4u * nbw + 32u * Fp8 + (Ks + 1u) * width, 64u);
+    c.f_ks[t] = Ks | (Ka << 16);
+    c.f_var_bytes[t] = round_up_u32(4u * nbw + 64u * Fp8 + (Ks + 1u) * width, 64u);
   }
 }
 
