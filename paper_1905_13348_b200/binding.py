@@ -171,4 +171,4 @@ def infaas_tally_static(d_decision, n_variants: int, d_count, d_counters, n=None
         raise ValueError("d_count is shorter than n_variants")
     _check(_load().infaas_tally_static(_dev_ptr(d_decision, "u32"), n, int(n_variants),
                                        _dev_ptr(d_count, "u32"), d_counters.data_ptr(),
-                                       d_count.device.index, _stream_ptr(stream)), "infaas_tally_static", "infaas_catalog_get_info")
+                                       d_count.device.index, _stream_ptr(stream)), "infaas_tally_static")

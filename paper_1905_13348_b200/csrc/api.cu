@@ -155,8 +155,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
   const size_t o_regions = carve((size_t)region_bytes);
-  const size_t o_flen = carve((size_t)n_tasks * 4), o_fks = carve((size_t)n_tasks * 4);
-  const size_t o_fvar = carve((size_t)n_tasks * 4), o_fhdr = carve((size_t)n_tasks * 8);
+  const size_t o_flen = carve((size_t)n_tasks * 4), o_fslow = carve((size_t)n_tasks * 8);
+  const size_t o_fvar = carve((size_t)n_tasks * 4), o_fhdr = carve((size_t)n_tasks * 16);
   const size_t o_image = carve((size_t)worst_image), o_hdr = carve(16);
   const size_t o_counters = carve(24), o_done = carve(4), o_err = carve(4);
 
@@ -198,9 +198,9 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.count_by_id = reinterpret_cast<uint32_t *>(base + o_count);
   d.regions = base + o_regions;
   d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
-  d.f_ks = reinterpret_cast<uint32_t *>(base + o_fks);
+  d.f_slow = reinterpret_cast<uint2 *>(base + o_fslow);
   d.f_var_bytes = reinterpret_cast<uint32_t *>(base + o_fvar);
-  d.f_hdr = reinterpret_cast<infaas::TaskHdr *>(base + o_fhdr);
+  d.f_hdr = reinterpret_cast<uint4 *>(base + o_fhdr);
   d.image = base + o_image;
   d.image_capacity = (uint32_t)worst_image;
   d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);

@@ -22,75 +22,78 @@ namespace infaas {
 // r comes from a table of SLO_BUCKETS records indexed by a monotone bucket of slo (top bits
 // of slo converted to float, shifted by `sh`, relative to `bmin`); a record holds the rank
 // below the bucket and the one distinct value inside it (as a 24-bit offset from the
-// bucket's smallest slo); a bucket with two or more values is flagged and its record gives
-// the range of Pd to compare against instead.  k comes from a bitmap over acc values with
-// running popcounts (24 bitmap bits + 8 prefix bits per word), exact at one basis point.
+// bucket's smallest slo).  A bucket holding two or more values sends the query to two
+// extra rows of T2 that contain only 0xFF, i.e. to the exact slow path.  k comes from a
+// bitmap over acc values with running popcounts (24 bitmap bits + 8 prefix bits per word),
+// exact at one basis point.
 //
 // Image (what the selection kernel stages in shared memory), all parts 64-byte aligned:
-//   hdr   u64[n_tasks]            per-task packed parameters (TaskHdr below)
-//   slo   u32[n_tasks][SLO_BUCKETS]   SLO records: lb << 24 | delta, or flagged:
-//                                     0xFF << 24 | lb << 8 | number of values in the bucket
-//   var   per-task blocks back to back, each: ids u32[8*Fp8], Pd u32[8*Fp8],
-//         acc bitmap u32[nbw], T2 u8[(Ks+1)*width], padded to 64 bytes
+//   hdr    uint4[n_tasks + 1]   fast-path parameters (below); entry n_tasks serves queries
+//                               whose task is out of range
+//   slow   uint2[n_tasks + 1]   slow-path parameters: aux offset, F | Ks<<8 | Ka<<16
+//   slo    u32[n_tasks + 1][SLO_BUCKETS]   SLO records: lb << 24 | delta
+//   dummy  64 bytes of 0x00, 64 bytes of 0xFF   (what tasks without an index point at)
+//   var    per-task blocks back to back, each:
+//          ids u32[8*Fp8], Pd u32[8*Fp8], acc bitmap u32[nbw], T2 u8[(Ks+3)*width],
+//          aux (what the nearest-miss search reads, see AuxLayout), padded to 64 bytes
 //
-// Cold data (read from global memory by the slow path only), per task in its region, V =
-// number of the task's variants:
-//   keys u64[V] (F used)  pred_lat | acc_bp << 32 in scan order;  ids u32[V] (F used);
-//   then, for an indexed list (Fi = min(V, INDEX_MAX_F)), what the nearest-miss search uses:
-//   bestA u8[Fi+1]   bestA[r]: position of the highest accuracy among the r smallest latencies
-//   bestB u8[Fi+1]   bestB[k]: position of the lowest latency among all but the k smallest accuracies
-//   order u8[Fi]     positions sorted by latency rank;  ordStart u8[Fi+1]: first index of rank r
-//   idxA u8[Fi], idxP u8[Fi]   accuracy / latency rank of each position
-//   then, 64-byte aligned, the var block before it is packed into the image
+// hdr words (offsets are bytes from the start of the image, 18 bits):
+//   x = ids_off | acc_min << 18            y = bitmap_off | width << 18
+//   z = t2_off | sh << 18 | flags << 21    w = bmin | x_max << 15     (x_max = 24*nbw - 1)
+//
+// Per task in its region (global memory): keys u64[V] (pred_lat | acc_bp << 32, scan
+// order, F used), ids u32[V]; then, 64-byte aligned, the var block before it is packed.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
 constexpr uint32_t ACC_WORD_BITS = 24;
 constexpr uint32_t MAX_ACC_WORDS = 420;          // covers 0..10000 bp at 24 per word
-constexpr uint32_t SLO_FLAGGED = 0xFFu;
-constexpr uint32_t VB_NOT_INDEXED = 0xFFEu;      // hdr.var_base value: list too long for the index
-constexpr uint32_t VB_NO_VARIANTS = 0xFFFu;      // hdr.var_base value: the task has no variant
-
-// hdr word 0: var_base (12 bits, units of 64 B from the start of the var section)
-//             | acc_min4 << 12 (12 bits, units of 4 bp) | sh << 24 (3 bits) | Fp8 << 27 (5 bits)
-// hdr word 1: bmin (15 bits) | nbw << 15 (9 bits) | width2 << 24 (7 bits, units of 2)
-struct TaskHdr {
-  uint32_t w0, w1;
-};
+constexpr uint32_t IMAGE_OFFSET_LIMIT = 1u << 18;
+constexpr uint32_t HDR_FLAG_INVALID = 1u;        // no variant (or task out of range): answer INVALID
+constexpr uint32_t HDR_FLAG_NOT_INDEXED = 2u;    // list without index: the slow path walks it
 
 inline __host__ __device__ uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-inline __host__ __device__ uint32_t image_slo_offset(uint32_t n_tasks) { return round_up_u32(8u * n_tasks, 64u); }
-inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) {
-  return image_slo_offset(n_tasks) + 4u * SLO_BUCKETS * n_tasks;
+inline __host__ __device__ uint32_t image_slow_offset(uint32_t n_tasks) { return round_up_u32(16u * (n_tasks + 1u), 64u); }
+inline __host__ __device__ uint32_t image_slo_offset(uint32_t n_tasks) {
+  return image_slow_offset(n_tasks) + round_up_u32(8u * (n_tasks + 1u), 64u);
 }
+inline __host__ __device__ uint32_t image_dummy_offset(uint32_t n_tasks) {
+  return image_slo_offset(n_tasks) + 4u * SLO_BUCKETS * (n_tasks + 1u);
+}
+inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) { return image_dummy_offset(n_tasks) + 128u; }
 
-// Worst-case bytes of one task's var block and of its region (cold data + var block).
-inline __host__ __device__ uint32_t var_capacity(uint32_t V) {
-  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
-  return round_up_u32(4u * MAX_ACC_WORDS + 8u * round_up_u32(F, 8) + (F + 1u) * (F + 2u), 64u);
-}
-struct ColdLayout {    // byte offsets inside a task's region
-  uint32_t keys, ids, bestA, bestB, order, ordStart, idxA, idxP, var;
+// Byte offsets inside the aux part of a var block, for a list of F entries with Ks / Ka
+// distinct latencies / accuracies.
+//   bestA[r], r in 0..Ks: position of the highest accuracy among the r smallest latencies
+//   bestB[k], k in 0..Ka: position of the lowest latency among all but the k smallest accuracies
+//   order[o]: positions sorted by latency rank; ordRank[o]: that rank; ordStart[r]: first o of rank r
+//   idxA[p], idxP[p]: accuracy / latency rank of position p;  Ad u16[Ka]: distinct accuracies
+struct AuxLayout {
+  uint32_t bestA, bestB, order, ordRank, ordStart, idxA, idxP, Ad, bytes;
 };
-inline __host__ __device__ ColdLayout cold_layout(uint32_t V) {
-  const uint32_t Fi = V < INDEX_MAX_F ? V : INDEX_MAX_F;
-  ColdLayout L;
-  L.keys = 0;
-  L.ids = 8u * V;
-  L.bestA = 12u * V;
-  L.bestB = L.bestA + Fi + 1u;
-  L.order = L.bestB + Fi + 1u;
-  L.ordStart = L.order + Fi;
-  L.idxA = L.ordStart + Fi + 1u;
-  L.idxP = L.idxA + Fi;
-  L.var = round_up_u32(L.idxP + Fi, 64u);
+inline __host__ __device__ AuxLayout aux_layout(uint32_t F, uint32_t Ks, uint32_t Ka) {
+  AuxLayout L;
+  L.bestA = 0;
+  L.bestB = L.bestA + Ks + 1u;
+  L.order = L.bestB + Ka + 1u;
+  L.ordRank = L.order + F;
+  L.ordStart = L.ordRank + F;
+  L.idxA = L.ordStart + Ks + 1u;
+  L.idxP = L.idxA + F;
+  L.Ad = (L.idxP + F + 1u) & ~1u;
+  L.bytes = L.Ad + 2u * Ka;
   return L;
 }
-inline __host__ __device__ uint32_t region_var_offset(uint32_t V) { return cold_layout(V).var; }
-inline __host__ __device__ uint32_t region_capacity(uint32_t V) {
-  return region_var_offset(V) + var_capacity(V);
+
+// Worst-case bytes of one task's var block and of its region.
+inline __host__ __device__ uint32_t var_capacity(uint32_t V) {
+  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
+  return round_up_u32(8u * round_up_u32(F, 8) + 4u * MAX_ACC_WORDS + (F + 3u) * (F + 2u) +
+                          aux_layout(F, F, F).bytes, 64u);
 }
+inline __host__ __device__ uint32_t region_var_offset(uint32_t V) { return round_up_u32(12u * V, 64u); }
+inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return region_var_offset(V) + var_capacity(V); }
 
 // ---------------------------------------------------------------------------------------
 // Device catalog.  "Slot" order: variants bucketed by task, ascending id inside a task;
@@ -113,11 +116,11 @@ struct DeviceCatalog {
   unsigned long long *s_served;
   uint32_t *count_by_id;     // [n_variants], zero between windows
 
-  unsigned char *regions;    // per task: keys, Pd, then the var block before packing
+  unsigned char *regions;    // per task: keys, ids, then the var block before packing
   uint32_t *f_len;           // [n_tasks] list length F
-  uint32_t *f_ks;            // [n_tasks] Ks | Ka << 16: distinct pred_lat / acc_bp values (0 if not indexed)
   uint32_t *f_var_bytes;     // [n_tasks] bytes of the task's var block (0 if not indexed)
-  TaskHdr *f_hdr;            // [n_tasks] header words without var_base (filled in when packing)
+  uint4 *f_hdr;              // [n_tasks] hdr words with offsets relative to the var block
+  uint2 *f_slow;             // [n_tasks] slow words, aux offset relative to the var block
 
   unsigned char *image;      // packed image, image_capacity bytes, 256-byte aligned
   uint32_t image_capacity;
@@ -150,11 +153,11 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream);
 cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uint64_t n,
                          cudaStream_t stream);
+// Shared memory the launcher actually reserves for the image when asked for `image_smem`.
+uint32_t select_image_smem(uint32_t image_smem);
 // `image_smem`: bytes of dynamic shared memory reserved for the staged image (multiple of
 // 16).  If the image is larger at run time the kernel reads it from global memory instead.
 // Returns cudaErrorInvalidValue if n is too large for the launch geometry.
-// Shared memory the launcher actually reserves for the image when asked for `image_smem`.
-uint32_t select_image_smem(uint32_t image_smem);
 cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const uint32_t *d_slo,
                           const uint16_t *d_min_acc, uint64_t n, uint32_t *d_decision,
                           int sm_count, uint32_t image_smem, cudaStream_t stream);

@@ -78,8 +78,16 @@ struct SharedImage {
   __device__ __forceinline__ uint32_t u32(uint32_t off) const {
     uint32_t v; asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
   }
+  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
+    uint32_t v; asm("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
+  }
   __device__ __forceinline__ uint2 v2(uint32_t off) const {
     uint2 v; asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(base + off)); return v;
+  }
+  __device__ __forceinline__ uint4 v4(uint32_t off) const {
+    uint4 v;
+    asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(base + off));
+    return v;
   }
 };
 
@@ -89,141 +97,127 @@ struct GlobalImage {
   __device__ __forceinline__ uint32_t u32(uint32_t off) const {
     return __ldg(reinterpret_cast<const uint32_t *>(base + off));
   }
+  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
+    return __ldg(reinterpret_cast<const uint16_t *>(base + off));
+  }
   __device__ __forceinline__ uint2 v2(uint32_t off) const {
     return __ldg(reinterpret_cast<const uint2 *>(base + off));
   }
-};
-
-// Per-task parameters unpacked from the two header words (see common.cuh).
-struct TaskParams {
-  uint32_t vb, acc_min, sh, ids_off, pd_off, bitmap_off, t2_off, bmin, nbw, width;
-};
-__device__ __forceinline__ TaskParams unpack_hdr(uint32_t w0, uint32_t w1, uint32_t var0) {
-  TaskParams P;
-  P.vb = w0 & 0xFFFu;
-  P.acc_min = ((w0 >> 12) & 0xFFFu) << 2;
-  P.sh = (w0 >> 24) & 7u;
-  P.bmin = w1 & 0x7FFFu;
-  P.nbw = (w1 >> 15) & 0x1FFu;
-  P.width = ((w1 >> 24) & 0x7Fu) << 1;
-  P.ids_off = var0 + (P.vb << 6);
-  P.pd_off = P.ids_off + ((w0 >> 27) << 5);
-  P.bitmap_off = P.pd_off + ((w0 >> 27) << 5);
-  P.t2_off = P.bitmap_off + (P.nbw << 2);
-  return P;
-}
-
-// r = #{distinct list latencies <= slo}: one bucket record and one comparison; a flagged
-// bucket (two or more values inside) compares against that short range of Pd instead.
-template <class Img>
-__device__ __forceinline__ uint32_t slo_rank(const Img &img, const TaskParams &P, uint32_t slo_off,
-                                             uint32_t task, uint32_t slo) {
-  const uint32_t b = (__float_as_uint(__uint2float_rz(slo)) >> 16) >> P.sh;
-  const uint32_t j = min(max(b, P.bmin) - P.bmin, SLO_BUCKETS - 1u);
-  const uint32_t lo = j ? __float2uint_ru(__uint_as_float(((P.bmin + j) << P.sh) << 16)) : 0u;
-  const uint32_t rec = img.u32(slo_off + ((task * SLO_BUCKETS + j) << 2));
-  uint32_t r = (rec >> 24) + ((slo - lo) >= (rec & 0x00FFFFFFu));
-  if ((rec >> 24) == SLO_FLAGGED) {
-    r = (rec >> 8) & 0xFFFFu;
-    const uint32_t end = r + (rec & 0xFFu);
-    for (uint32_t i = r; i < end; ++i) r += img.u32(P.pd_off + (i << 2)) <= slo;
+  __device__ __forceinline__ uint4 v4(uint32_t off) const {
+    return __ldg(reinterpret_cast<const uint4 *>(base + off));
   }
-  return r;
-}
+};
 
 // k = #{distinct list accuracies < min_acc}, from the bitmap with running popcounts.
 template <class Img>
-__device__ __forceinline__ uint32_t acc_rank(const Img &img, const TaskParams &P, uint32_t min_acc) {
-  const uint32_t x = min(max(min_acc, P.acc_min) - P.acc_min, ACC_WORD_BITS * P.nbw - 1u);
+__device__ __forceinline__ uint32_t acc_rank(const Img &img, uint32_t bitmap_off, uint32_t acc_min,
+                                             uint32_t x_max, uint32_t min_acc) {
+  const uint32_t x = min(max(min_acc, acc_min) - acc_min, x_max);
   const uint32_t w = (x * 43691u) >> 20;                    // x / 24 for x < 2^16
-  const uint32_t word = img.u32(P.bitmap_off + (w << 2));
+  const uint32_t word = img.u32(bitmap_off + (w << 2));
   return (word >> 24) + __popc(word & ((1u << (x - w * ACC_WORD_BITS)) - 1u));
 }
 
-// Fast path: the decision, INFAAS_INVALID, or PENDING when nothing is feasible or the
-// task's list has no index (the parked query is then resolved by decide_slow).
+// Fast path, straight-line: five loads.  Returns the decision, INFAAS_INVALID, or PENDING
+// when the query needs the slow path: nothing feasible, an SLO bucket with several values,
+// or a task whose list has no index (those read 0xFF from T2 by construction).
 template <class Img>
 __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks, uint32_t slo_off,
-                                                uint32_t var0, uint32_t task, uint32_t slo,
-                                                uint32_t min_acc) {
-  if (task >= n_tasks) return INFAAS_INVALID;
-  const uint2 h = img.v2(task << 3);
-  const TaskParams P = unpack_hdr(h.x, h.y, var0);
-  if (P.vb >= VB_NOT_INDEXED) return P.vb == VB_NO_VARIANTS ? INFAAS_INVALID : PENDING;
-  const uint32_t r = slo_rank(img, P, slo_off, task, slo);
-  const uint32_t k = acc_rank(img, P, min_acc);
-  const uint32_t pos = img.u8(P.t2_off + r * P.width + k);
-  if (pos == 0xFFu) return PENDING;
-  return img.u32(P.ids_off + (pos << 2));
+                                                uint32_t task, uint32_t slo, uint32_t min_acc) {
+  const uint32_t t = min(task, n_tasks);
+  const uint4 h = img.v4(t << 4);
+  const uint32_t sh = (h.z >> 18) & 7u, bmin = h.w & 0x7FFFu;
+  // r = #{distinct list latencies <= slo}: bucket record + one comparison
+  const uint32_t b = (__float_as_uint(__uint2float_rz(slo)) >> 16) >> sh;
+  const uint32_t j = min(max(b, bmin) - bmin, SLO_BUCKETS - 1u);
+  const uint32_t lo = j ? __float2uint_ru(__uint_as_float((bmin + j) << (sh + 16u))) : 0u;
+  const uint32_t rec = img.u32(slo_off + (((t << 8) + j) << 2));
+  const uint32_t r = (rec >> 24) + ((slo - lo) >= (rec & 0x00FFFFFFu));
+  const uint32_t k = acc_rank(img, h.y & 0x3FFFFu, h.x >> 18, h.w >> 15, min_acc);
+  const uint32_t pos = img.u8((h.z & 0x3FFFFu) + r * (h.y >> 18) + k);
+  const bool none = pos == 0xFFu;
+  const uint32_t id = img.u32((h.x & 0x3FFFFu) + (none ? 0u : pos << 2));
+  return none ? (((h.z >> 21) & HDR_FLAG_INVALID) ? INFAAS_INVALID : PENDING) : id;
 }
 
-// d = 10^4 * over_lat + slo * under_acc of one list entry (64-bit).
-__device__ __forceinline__ unsigned long long miss_distance(unsigned long long key, uint32_t slo,
+// d = 10^4 * over_lat + slo * under_acc (64-bit).
+__device__ __forceinline__ unsigned long long miss_distance(uint32_t pred, uint32_t acc, uint32_t slo,
                                                             uint32_t min_acc) {
-  const uint32_t pred = (uint32_t)key, acc = (uint32_t)(key >> 32);
   const uint32_t over = pred > slo ? pred - slo : 0u;
   const uint32_t under = min_acc > acc ? min_acc - acc : 0u;
   return (unsigned long long)over * 10000ull + (unsigned long long)slo * under;
 }
 
-// Slow path for a parked query.  The nearest miss is the entry smallest in (d, position):
-// position order is (cost, pred_lat, -acc, id) order.  Cold data comes from the task's
-// region in global memory.
-//   Indexed list: nothing is feasible (the fast path said so).  Entries that meet the SLO
-//   all miss the accuracy, and the best of them is the one with the highest accuracy
-//   (bestA); entries that meet the accuracy all miss the SLO, the best being the one with
-//   the lowest latency (bestB); an entry that misses both can only win if its accuracy is
-//   above bestA's and its latency not above bestB's, so only that rank rectangle is walked.
-//   List without index: walk it, first for a feasible entry, then for the distance.
+// Slow path for a parked query (never an invalid one).
+//   Indexed list: exact ranks (binary search over Pd), then T2.  If nothing is feasible the
+//   nearest miss is the entry smallest in (d, position) -- position order is (cost,
+//   pred_lat, -acc, id) order.  Entries that meet the SLO all miss the accuracy, the best
+//   of them is the one with the highest accuracy (bestA); entries that meet the accuracy
+//   all miss the SLO, the best being the one with the lowest latency (bestB); an entry
+//   that misses both can only win with accuracy above bestA's, latency not above bestB's
+//   and a latency overshoot that alone stays below the best distance so far, so the walk
+//   in latency order stops early.
+//   List without index: walk it in global memory, for a feasible entry, then for the distance.
 template <class Img>
-__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t slo_off,
-                                                uint32_t var0, uint32_t task, uint32_t slo,
-                                                uint32_t min_acc) {
-  const uint32_t F = __ldg(c.f_len + task);
-  const uint32_t V = __ldg(c.task_off + task + 1) - __ldg(c.task_off + task);
-  const unsigned char *region = c.regions + __ldg(c.reg_off + task);
-  const ColdLayout CL = cold_layout(V);
-  const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(region);
-  const uint32_t *ids = reinterpret_cast<const uint32_t *>(region + CL.ids);
-  const uint2 h = img.v2(task << 3);
-  const TaskParams P = unpack_hdr(h.x, h.y, var0);
+__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t task,
+                                                uint32_t slo, uint32_t min_acc) {
+  const uint4 h = img.v4(task << 4);
   unsigned long long best = ~0ull;
   uint32_t best_i = 0;
-  if (P.vb < VB_NOT_INDEXED) {
-    const uint32_t kk = __ldg(c.f_ks + task), Ks = kk & 0xFFFFu, Ka = kk >> 16;
-    const uint32_t r = slo_rank(img, P, slo_off, task, slo);
-    const uint32_t k = acc_rank(img, P, min_acc);
+  if (!((h.z >> 21) & HDR_FLAG_NOT_INDEXED)) {
+    const uint2 sl = img.v2(image_slow_offset(c.n_tasks) + (task << 3));
+    const uint32_t F = sl.y & 0xFFu, Ks = (sl.y >> 8) & 0xFFu, Ka = sl.y >> 16;
+    const uint32_t ids_off = h.x & 0x3FFFFu, pd_off = ids_off + (((F + 7u) >> 3) << 5);
+    const AuxLayout AL = aux_layout(F, Ks, Ka);
+    const uint32_t aux = sl.x;
+    uint32_t lo = 0, hi = Ks;                              // r = #{Pd <= slo}
+    while (lo < hi) {
+      const uint32_t mid = (lo + hi) >> 1;
+      if (img.u32(pd_off + (mid << 2)) <= slo) lo = mid + 1; else hi = mid;
+    }
+    const uint32_t r = lo;
+    const uint32_t k = acc_rank(img, h.y & 0x3FFFFu, h.x >> 18, h.w >> 15, min_acc);
+    const uint32_t pos = img.u8((h.z & 0x3FFFFu) + r * (h.y >> 18) + k);
+    if (pos != 0xFFu) return img.u32(ids_off + (pos << 2));
     uint32_t acc_rank_floor = 0;          // candidates need accuracy rank >= this
     uint32_t lat_rank_cap = Ks;           // ... and latency rank < this
-    if (r > 0) {                          // some entry meets the SLO
-      const uint32_t pA = __ldg(region + CL.bestA + r);
-      best = miss_distance(__ldg(keys + pA), slo, min_acc);
+    if (r > 0) {                          // some entry meets the SLO (and misses the accuracy)
+      const uint32_t pA = img.u8(aux + AL.bestA + r), ia = img.u8(aux + AL.idxA + pA);
+      best = (unsigned long long)slo * (min_acc - img.u16(aux + AL.Ad + (ia << 1)));
       best_i = pA;
-      acc_rank_floor = __ldg(region + CL.idxA + pA) + 1u;
+      acc_rank_floor = ia + 1u;
     }
-    if (k < Ka) {                         // some entry meets the accuracy
-      const uint32_t pB = __ldg(region + CL.bestB + k);
-      const unsigned long long d = miss_distance(__ldg(keys + pB), slo, min_acc);
+    if (k < Ka) {                         // some entry meets the accuracy (and misses the SLO)
+      const uint32_t pB = img.u8(aux + AL.bestB + k), ip = img.u8(aux + AL.idxP + pB);
+      const unsigned long long d = (unsigned long long)(img.u32(pd_off + (ip << 2)) - slo) * 10000ull;
       if (d < best || (d == best && pB < best_i)) { best = d; best_i = pB; }
-      lat_rank_cap = __ldg(region + CL.idxP + pB) + 1u;
+      lat_rank_cap = ip + 1u;
     }
-    for (uint32_t o = __ldg(region + CL.ordStart + r); o < F; ++o) {   // latency ranks >= r
-      const uint32_t p = __ldg(region + CL.order + o);
-      if (__ldg(region + CL.idxP + p) >= lat_rank_cap) break;
-      const uint32_t ia = __ldg(region + CL.idxA + p);
+    for (uint32_t o = img.u8(aux + AL.ordStart + r); o < F; ++o) {   // latency ranks >= r
+      const uint32_t ip = img.u8(aux + AL.ordRank + o);
+      if (ip >= lat_rank_cap) break;
+      const unsigned long long over = (unsigned long long)(img.u32(pd_off + (ip << 2)) - slo) * 10000ull;
+      if (over > best) break;             // later entries overshoot the SLO even more
+      const uint32_t p = img.u8(aux + AL.order + o), ia = img.u8(aux + AL.idxA + p);
       if (ia >= acc_rank_floor && ia < k) {
-        const unsigned long long d = miss_distance(__ldg(keys + p), slo, min_acc);
+        const unsigned long long d = over + (unsigned long long)slo * (min_acc - img.u16(aux + AL.Ad + (ia << 1)));
         if (d < best || (d == best && p < best_i)) { best = d; best_i = p; }
       }
     }
-    return INFAAS_NO_FEASIBLE | __ldg(ids + best_i);
+    return INFAAS_NO_FEASIBLE | img.u32(ids_off + (best_i << 2));
   }
+  const uint32_t F = __ldg(c.f_len + task);
+  const uint32_t V = __ldg(c.task_off + task + 1) - __ldg(c.task_off + task);
+  const unsigned char *region = c.regions + __ldg(c.reg_off + task);
+  const unsigned long long *keys = reinterpret_cast<const unsigned long long *>(region);
+  const uint32_t *ids = reinterpret_cast<const uint32_t *>(region + 8u * V);
   for (uint32_t i = 0; i < F; ++i) {
     const unsigned long long e = __ldg(keys + i);
     if ((uint32_t)e <= slo && (uint32_t)(e >> 32) >= min_acc) return __ldg(ids + i);
   }
   for (uint32_t i = 0; i < F; ++i) {
-    const unsigned long long d = miss_distance(__ldg(keys + i), slo, min_acc);
+    const unsigned long long e = __ldg(keys + i);
+    const unsigned long long d = miss_distance((uint32_t)e, (uint32_t)(e >> 32), slo, min_acc);
     if (d < best) { best = d; best_i = i; }
   }
   return INFAAS_NO_FEASIBLE | __ldg(ids + best_i);
@@ -238,13 +232,13 @@ struct Queries {
 
 // Resolve up to 32 parked queries, one per lane.  `rel` is the query's offset from `q0`.
 template <class Img>
-__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, uint32_t slo_off,
-                                               uint32_t var0, const Queries &q, uint64_t q0, const uint32_t *park,
-                                               uint32_t first, uint32_t count) {
+__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, const Queries &q,
+                                               uint64_t q0, const uint32_t *park, uint32_t first,
+                                               uint32_t count) {
   const uint32_t lane = threadIdx.x & 31;
   if (lane < count) {
     const uint64_t i = q0 + park[first + lane];
-    q.decision[i] = decide_slow(img, c, slo_off, var0, q.task[i], q.slo[i], q.min_acc[i]);
+    q.decision[i] = decide_slow(img, c, q.task[i], q.slo[i], q.min_acc[i]);
   }
 }
 
@@ -259,7 +253,7 @@ template <class Img>
 __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
                                             uint64_t n, uint64_t per_cta, uint32_t *park_all) {
   const uint32_t n_tasks = c.n_tasks;
-  const uint32_t slo_off = image_slo_offset(n_tasks), var0 = image_var_offset(n_tasks);
+  const uint32_t slo_off = image_slo_offset(n_tasks);
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   uint32_t *park = park_all + warp * PARK_CAP;
   uint32_t parked = 0;
@@ -290,10 +284,10 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
       a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
     }
     uint4 d;
-    d.x = decide_fast(img, n_tasks, slo_off, var0, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
-    d.y = decide_fast(img, n_tasks, slo_off, var0, t.x >> 16, s.y, a.x >> 16);
-    d.z = decide_fast(img, n_tasks, slo_off, var0, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
-    d.w = decide_fast(img, n_tasks, slo_off, var0, t.y >> 16, s.w, a.y >> 16);
+    d.x = decide_fast(img, n_tasks, slo_off, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
+    d.y = decide_fast(img, n_tasks, slo_off, t.x >> 16, s.y, a.x >> 16);
+    d.z = decide_fast(img, n_tasks, slo_off, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
+    d.w = decide_fast(img, n_tasks, slo_off, t.y >> 16, s.w, a.y >> 16);
     const uint32_t rel = (uint32_t)(tile * WARP_TILE) + lane * 4u;
     uint32_t *out = q.decision + q0 + rel;
     const bool any_pending = d.x == PENDING || d.y == PENDING || d.z == PENDING || d.w == PENDING;
@@ -313,7 +307,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
       __syncwarp();
       while (parked >= 32) {
         parked -= 32;
-        resolve_parked(img, c, slo_off, var0, q, q0, park, parked, 32);
+        resolve_parked(img, c, q, q0, park, parked, 32);
       }
       __syncwarp();
     }
@@ -326,7 +320,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
       uint32_t d = 0;
       if (rel < span) {
         const uint64_t i = q0 + rel;
-        d = decide_fast(img, n_tasks, slo_off, var0, q.task[i], q.slo[i], q.min_acc[i]);
+        d = decide_fast(img, n_tasks, slo_off, q.task[i], q.slo[i], q.min_acc[i]);
         if (d != PENDING) q.decision[i] = d;
       }
       park_append(park, parked, rel < span && d == PENDING, (uint32_t)rel);
@@ -334,11 +328,11 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
     __syncwarp();
     while (parked >= 32) {
       parked -= 32;
-      resolve_parked(img, c, slo_off, var0, q, q0, park, parked, 32);
+      resolve_parked(img, c, q, q0, park, parked, 32);
     }
   }
   __syncwarp();
-  resolve_parked(img, c, slo_off, var0, q, q0, park, 0, parked);
+  resolve_parked(img, c, q, q0, park, 0, parked);
 }
 
 __global__ void __launch_bounds__(SELECT_THREADS, 1)

@@ -162,8 +162,8 @@ struct IndexScratch {          // shared memory used while building one task's i
 
 // Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh).
 // S.pred / S.acc hold the list in scan order.  Writes the SLO records straight into the
-// image, the var block and the cold Pd array into the task's region, and the task's header
-// words (without var_base), Ks and var-block size into the per-task arrays.
+// image, the var block into the task's region, and the task's header words (offsets
+// relative to the var block) and var-block size into the per-task arrays.
 __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint32_t V, IndexScratch &S) {
   const uint32_t tid = threadIdx.x, B = blockDim.x;
   unsigned char *region = c.regions + c.reg_off[t];
@@ -201,16 +201,28 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     S.order[o] = (unsigned char)p;
   }
   __syncthreads();
-  const ColdLayout CL = cold_layout(V);
+
+  // var block layout
   const uint32_t Fp8 = (F + 7u) / 8u;
-  unsigned char *var = region + CL.var;
-  uint32_t *Pd_hot = reinterpret_cast<uint32_t *>(var + 32u * Fp8);
+  const uint32_t acc_min = S.Ad[0] & ~3u;
+  const uint32_t nbw = (S.Ad[Ka - 1] - acc_min + 2u + ACC_WORD_BITS - 1u) / ACC_WORD_BITS;
+  const uint32_t width = Ka + 1u;
+  const uint32_t off_pd = 32u * Fp8, off_bitmap = 64u * Fp8, off_t2 = off_bitmap + 4u * nbw;
+  const uint32_t off_aux = (off_t2 + (Ks + 3u) * width + 3u) & ~3u;
+  const AuxLayout AL = aux_layout(F, Ks, Ka);
+  unsigned char *var = region + region_var_offset(V);
+  unsigned char *aux = var + off_aux;
+
+  uint32_t *Pd_hot = reinterpret_cast<uint32_t *>(var + off_pd);
   for (uint32_t i = tid; i < Ks; i += B) Pd_hot[i] = S.Pd[i];
-  // what the nearest-miss search reads (cold)
+  uint16_t *Ad_hot = reinterpret_cast<uint16_t *>(aux + AL.Ad);
+  for (uint32_t i = tid; i < Ka; i += B) Ad_hot[i] = S.Ad[i];
+  // what the nearest-miss search reads
   for (uint32_t p = tid; p < F; p += B) {
-    region[CL.order + p] = S.order[p];
-    region[CL.idxA + p] = S.idxA[p];
-    region[CL.idxP + p] = S.idxP[p];
+    aux[AL.order + p] = S.order[p];
+    aux[AL.ordRank + p] = S.idxP[S.order[p]];
+    aux[AL.idxA + p] = S.idxA[p];
+    aux[AL.idxP + p] = S.idxP[p];
   }
   for (uint32_t r = tid; r <= Ks; r += B) {
     uint32_t best = 0xFFu, best_acc = 0, cnt = 0;           // highest accuracy among ranks < r
@@ -220,18 +232,19 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
         if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
       }
     }
-    region[CL.bestA + r] = (unsigned char)best;
-    region[CL.ordStart + r] = (unsigned char)cnt;
+    aux[AL.bestA + r] = (unsigned char)best;
+    aux[AL.ordStart + r] = (unsigned char)cnt;
   }
   for (uint32_t k = tid; k <= Ka; k += B) {
     uint32_t best = 0xFFu, best_pred = 0;                    // lowest latency among accuracy ranks >= k
     for (uint32_t p = 0; p < F; ++p) {
       if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
     }
-    region[CL.bestB + k] = (unsigned char)best;
+    aux[AL.bestB + k] = (unsigned char)best;
   }
 
-  // SLO records
+  // SLO records.  A bucket with two or more values points at row Ks + 1 of T2 (rows Ks + 1
+  // and Ks + 2 hold only 0xFF), so such a query goes to the slow path.
   const uint32_t cmin = float_code(S.Pd[0]), cmax = float_code(S.Pd[Ks - 1]);
   uint32_t sh = 0;
   while ((cmax >> sh) - (cmin >> sh) > SLO_BUCKETS - 1) ++sh;
@@ -244,24 +257,19 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
       lb += b < j;
       if (b == j) { ++cnt; thr = S.Pd[i]; }
     }
-    uint32_t rec;
+    uint32_t rec = (Ks + 1u) << 24;                           // two or more values: slow path
     if (cnt == 0) {
-      rec = lb ? ((lb - 1) << 24) : 0x00FFFFFFu;   // "always one more than lb-1" / never (lb = 0)
+      rec = lb ? ((lb - 1u) << 24) : 0x00FFFFFFu;             // always one more than lb - 1 (lb = 0 cannot occur)
     } else if (cnt == 1) {
       const uint32_t lo = j ? float_code_floor((bmin + j) << sh) : 0u;
       const uint32_t delta = thr - lo;
-      rec = delta < 0x01000000u ? (lb << 24) | delta : (SLO_FLAGGED << 24) | (lb << 8) | 1u;
-    } else {
-      rec = (SLO_FLAGGED << 24) | (lb << 8) | cnt;
+      if (delta < 0x01000000u) rec = (lb << 24) | delta;
     }
     slo_rec[j] = rec;
   }
 
-  // var block: ids (already written by the caller), Pd (above), accuracy bitmap, T2
-  const uint32_t acc_min = S.Ad[0] & ~3u;
-  const uint32_t nbw = (S.Ad[Ka - 1] - acc_min + 2u + ACC_WORD_BITS - 1u) / ACC_WORD_BITS;
-  const uint32_t width = (Ka + 2u) & ~1u;                     // Ka + 1 rounded up to even
-  uint32_t *bitmap = reinterpret_cast<uint32_t *>(var + 64u * Fp8);
+  // accuracy bitmap
+  uint32_t *bitmap = reinterpret_cast<uint32_t *>(var + off_bitmap);
   for (uint32_t w = tid; w < nbw; w += B) {
     uint32_t bits = 0, prefix = 0;
     for (uint32_t i = 0; i < Ka; ++i) {
@@ -271,7 +279,8 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     }
     bitmap[w] = (prefix << 24) | bits;
   }
-  unsigned char *T2 = var + 64u * Fp8 + 4u * nbw;
+  // T2, one thread per accuracy rank k: walk the positions in latency-rank order
+  unsigned char *T2 = var + off_t2;
   for (uint32_t k = tid; k < width; k += B) {
     uint32_t cur = 0xFFu, o = 0;
     T2[k] = 0xFFu;                                             // r = 0: no latency is met
@@ -283,14 +292,14 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
       }
       T2[r * width + k] = (unsigned char)cur;
     }
+    T2[(Ks + 1u) * width + k] = 0xFFu;
+    T2[(Ks + 2u) * width + k] = 0xFFu;
   }
   if (tid == 0) {
-    TaskHdr h;
-    h.w0 = ((acc_min >> 2) << 12) | (sh << 24) | (Fp8 << 27);
-    h.w1 = bmin | (nbw << 15) | ((width >> 1) << 24);
-    c.f_hdr[t] = h;
-    c.f_ks[t] = Ks | (Ka << 16);
-    c.f_var_bytes[t] = round_up_u32(4u * nbw + 64u * Fp8 + (Ks + 1u) * width, 64u);
+    c.f_hdr[t] = make_uint4(0u | (acc_min << 18), off_bitmap | (width << 18), off_t2 | (sh << 18),
+                            bmin | ((ACC_WORD_BITS * nbw - 1u) << 15));
+    c.f_slow[t] = make_uint2(off_aux, F | (Ks << 8) | (Ka << 16));
+    c.f_var_bytes[t] = round_up_u32(off_aux + AL.bytes, 64u);
   }
 }
 
@@ -389,7 +398,7 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   const bool indexed = F > 0 && F <= INDEX_MAX_F;
   unsigned char *region = c.regions + c.reg_off[t];
 
-  // 4. compact into the task's region (scan order): cold keys and ids, and the var block's ids
+  // 4. compact into the task's region (scan order): keys and ids, and the var block's ids
   unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(region);
   uint32_t *ids_g = reinterpret_cast<uint32_t *>(region + 8u * V);
   uint32_t *var_ids = reinterpret_cast<uint32_t *>(region + region_var_offset(V));
@@ -412,8 +421,6 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   if (indexed) {
     build_index(c, t, F, V, S);
   } else if (tid == 0) {
-    c.f_hdr[t] = TaskHdr{0u, 0u};
-    c.f_ks[t] = 0;
     c.f_var_bytes[t] = 0;
   }
   if (tid == 0) c.f_len[t] = F;
@@ -430,8 +437,25 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   __threadfence();
 
   const uint32_t T = c.n_tasks;
-  TaskHdr *hdr = reinterpret_cast<TaskHdr *>(c.image);
-  const uint32_t var0 = image_var_offset(T);
+  uint4 *hdr = reinterpret_cast<uint4 *>(c.image);
+  uint2 *slow = reinterpret_cast<uint2 *>(c.image + image_slow_offset(T));
+  const uint32_t dummy = image_dummy_offset(T), var0 = image_var_offset(T);
+  // headers of a task without index: everything points at the dummy block, where the
+  // bitmap reads 0 and T2 reads 0xFF ("nothing found")
+  const uint4 dummy_hdr = make_uint4(dummy, dummy, dummy + 64u, 0u);
+  if (tid < 32) {                               // dummy block, the out-of-range entry and its SLO row
+    reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid < 16 ? 0u : 0xFFFFFFFFu;
+    if (tid == 0) {
+      uint4 h = dummy_hdr;
+      h.z |= HDR_FLAG_INVALID << 21;
+      hdr[T] = h;
+      slow[T] = make_uint2(0u, 0u);
+    }
+  }
+  {
+    uint32_t *row = reinterpret_cast<uint32_t *>(c.image + image_slo_offset(T)) + T * SLO_BUCKETS;
+    for (uint32_t j = tid; j < SLO_BUCKETS; j += B) row[j] = 0u;
+  }
   // 5a. var offsets = exclusive prefix sum of the var-block sizes (chunks of B tasks)
   uint32_t carry = 0, longest = 0, entries = 0, not_indexed = 0;
   __shared__ uint32_t scan_buf[1024];
@@ -440,9 +464,7 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   for (uint32_t t0 = 0; t0 < T; t0 += B) {
     const uint32_t tt = t0 + tid;
     const uint32_t len = tt < T ? __ldcg(c.f_len + tt) : 0u;
-    uint32_t vbytes = tt < T ? __ldcg(c.f_var_bytes + tt) : 0u;
-    // a block that would start beyond what var_base can address is left out: the task is
-    // then served by the slow path (decided per task below, after the scan)
+    const uint32_t vbytes = tt < T ? __ldcg(c.f_var_bytes + tt) : 0u;
     scan_buf[tid] = vbytes;
     __syncthreads();
     for (uint32_t o = 1; o < B; o <<= 1) {      // Hillis-Steele inclusive scan
@@ -455,32 +477,41 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
     const uint32_t incl = scan_buf[tid];
     __syncthreads();                                               // scan_buf is reused below
     if (var0 + carry + chunk_total > c.image_capacity) overflow = true;   // uniform
-    const uint32_t off = carry + incl - vbytes;                    // from the start of the var section
-    const bool addressable = (off >> 6) < VB_NOT_INDEXED;
+    const uint32_t off = var0 + carry + incl - vbytes;             // from the start of the image
+    // a block that does not end below what the 18-bit offsets can address is left out: the
+    // task is then served by the slow path, like one whose list is too long for the index
+    const bool addressable = off + vbytes <= IMAGE_OFFSET_LIMIT;
     if (tt < T && !overflow) {
-      const uint2 raw = __ldcg(reinterpret_cast<const uint2 *>(c.f_hdr + tt));
-      TaskHdr h{raw.x, raw.y};
-      uint32_t vb;
-      if (len == 0) vb = VB_NO_VARIANTS;
-      else if (vbytes == 0 || !addressable) vb = VB_NOT_INDEXED;
-      else vb = off >> 6;
-      h.w0 = (h.w0 & ~0xFFFu) | vb;
+      uint4 h = dummy_hdr;
+      uint2 sl = make_uint2(0u, len > 255u ? 0u : len);
+      if (len == 0) {
+        h.z |= HDR_FLAG_INVALID << 21;
+      } else if (vbytes == 0 || !addressable) {
+        h.z |= HDR_FLAG_NOT_INDEXED << 21;
+        ++not_indexed;
+      } else {
+        const uint4 rel = __ldcg(c.f_hdr + tt);
+        const uint2 srel = __ldcg(c.f_slow + tt);
+        h = make_uint4(rel.x + off, rel.y + off, rel.z + off, rel.w);
+        sl = make_uint2(srel.x + off, srel.y);
+      }
       hdr[tt] = h;
-      not_indexed += (vb == VB_NOT_INDEXED);
+      slow[tt] = sl;
     }
     // offsets stay ascending: empty blocks share the next block's offset, and the blocks
     // that are left out (and the padding past T) form a suffix of sentinels
     scan_buf[tid] = (tt < T && addressable) ? off : 0xFFFFFFFFu;
-    if (tid == 0) s_copy_end = carry;
+    if (tid == 0) s_copy_end = var0 + carry;
     __syncthreads();
     if (tt < T && addressable && vbytes) atomicMax(&s_copy_end, off + vbytes);
     __syncthreads();
     // 5b. copy this chunk's var blocks: 16-byte units spread over all threads; a unit finds
     // its block by binary search over the chunk's ascending offsets
     if (!overflow) {
-      const uint32_t units = (s_copy_end - carry) >> 4;
+      const uint32_t first = var0 + carry;
+      const uint32_t units = (s_copy_end - first) >> 4;
       const uint4 *reg4 = reinterpret_cast<const uint4 *>(c.regions);
-      uint4 *img4 = reinterpret_cast<uint4 *>(c.image + var0);
+      uint4 *img4 = reinterpret_cast<uint4 *>(c.image);
       for (uint32_t u0 = 0; u0 < units; u0 += 4u * B) {
         uint4 v[4];
         uint32_t dst[4];
@@ -489,19 +520,17 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
           const uint32_t u = u0 + (uint32_t)j * B + tid;
           dst[j] = 0xFFFFFFFFu;
           if (u < units) {
-            const uint32_t byte = carry + (u << 4);
+            const uint32_t byte = first + (u << 4);
             uint32_t lo = 0, hi = B;                    // last i with scan_buf[i] <= byte
             while (hi - lo > 1) {
               const uint32_t mid = (lo + hi) >> 1;
               if (scan_buf[mid] <= byte) lo = mid; else hi = mid;
             }
-            {
-              const uint32_t tsrc = t0 + lo;
-              const uint32_t Vt = __ldg(c.task_off + tsrc + 1) - __ldg(c.task_off + tsrc);
-              const uint32_t src_byte = __ldg(c.reg_off + tsrc) + region_var_offset(Vt) + (byte - scan_buf[lo]);
-              v[j] = __ldcg(reg4 + (src_byte >> 4));
-              dst[j] = byte >> 4;
-            }
+            const uint32_t tsrc = t0 + lo;
+            const uint32_t Vt = __ldg(c.task_off + tsrc + 1) - __ldg(c.task_off + tsrc);
+            const uint32_t src_byte = __ldg(c.reg_off + tsrc) + region_var_offset(Vt) + (byte - scan_buf[lo]);
+            v[j] = __ldcg(reg4 + (src_byte >> 4));
+            dst[j] = byte >> 4;
           }
         }
 #pragma unroll
