@@ -208,3 +208,79 @@ def test_alignment_and_null_errors():
         P.infaas_select_batch(cat, d_task, None, d_acc, d_dec, n=8)
     assert e.value.code == -1
     cat.free()
+
+
+# -- full sizes, in the launch configuration the benchmark times ----------------------------
+def _np_pred(rows, queued):
+    lat, q, b = (rows["lat_us"].astype(np.uint64), queued.astype(np.uint64),
+                 rows["batch"].astype(np.uint64))
+    return np.minimum(lat + q * lat // b, np.uint64(2**32 - 1)).astype(np.uint32)
+
+
+def _assert_state_fast(cat, o, rows):
+    import paper_1905_13348_b200 as P
+    st = P.infaas_catalog_get_state(cat)
+    assert np.array_equal(st["queued"], o.queued)
+    assert np.array_equal(st["pred_lat_us"], _np_pred(rows, o.queued))
+    assert np.array_equal(st["served_total"], o.served_total)
+    assert np.array_equal(st["counters"], o.counters)
+
+
+def _threads():
+    import os
+    return os.cpu_count() or 1
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C4"])
+def test_full_size_single_launch_then_update(name):
+    """All queries of the configuration in ONE infaas_select_batch (the launch shape the
+    benchmark times: one contiguous range per SM), then one load update over all decisions,
+    then a second launch against the updated load."""
+    import paper_1905_13348_b200 as P
+    w = W.make(name)
+    window_us = max(1, w.n_queries // max(1, w.window)) * w.window_us if w.window else 1_000_000
+    window_us = min(window_us, 2**32 - 1)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    try:
+        for rnd in range(2):
+            want = o.select(w.task, w.slo_us, w.min_acc_bp, _threads())
+            d_dec = gpu_select(cat, w.task, w.slo_us, w.min_acc_bp)
+            got = _to_host_u32(d_dec)
+            bad = np.flatnonzero(got != want)
+            assert bad.size == 0, (name, rnd, bad[:5], got[bad[:5]], want[bad[:5]])
+            P.infaas_load_update(cat, d_dec, window_us)
+            o.load_update(want, window_us)
+            _assert_state_fast(cat, o, w.rows)
+    finally:
+        cat.free()
+
+
+@pytest.mark.parametrize("name,state_every", [("C3", 16), ("C5", 100)])
+def test_full_size_windowed(name, state_every):
+    """The configuration as a stream of windows (select one window, update, repeat): every
+    decision of every window is compared; the load state every `state_every` windows and at
+    the end."""
+    import paper_1905_13348_b200 as P
+    torch = _torch()
+    w = W.make(name)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    d_task, d_slo, d_acc = _to_dev(w.task), _to_dev(w.slo_us), _to_dev(w.min_acc_bp)
+    d_dec = torch.empty(w.n_queries, dtype=torch.int32, device="cuda")
+    nwin = w.n_queries // w.window
+    try:
+        for k in range(nwin):
+            s = slice(k * w.window, (k + 1) * w.window)
+            P.infaas_select_batch(cat, d_task[s], d_slo[s], d_acc[s], d_dec[s])
+            P.infaas_load_update(cat, d_dec[s], w.window_us)
+            want = o.select(w.task[s], w.slo_us[s], w.min_acc_bp[s], _threads())
+            o.load_update(want, w.window_us)
+            got = _to_host_u32(d_dec[s])
+            bad = np.flatnonzero(got != want)
+            assert bad.size == 0, (name, k, bad[:5], got[bad[:5]], want[bad[:5]])
+            if (k + 1) % state_every == 0 or k == nwin - 1:
+                _assert_state_fast(cat, o, w.rows)
+        assert int(o.counters.sum()) == w.n_queries
+    finally:
+        cat.free()
