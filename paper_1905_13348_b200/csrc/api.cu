@@ -144,7 +144,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
 
   // ---- one arena, carved into 256-byte aligned arrays ----
   uint64_t worst_image = infaas::image_var_offset(n_tasks);
-  for (uint32_t t = 0; t < n_tasks; ++t) worst_image += infaas::var_capacity(task_off[t + 1] - task_off[t]);
+  for (uint32_t t = 0; t < n_tasks; ++t) worst_image += infaas::block_capacity(task_off[t + 1] - task_off[t]);
   if (worst_image > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
   size_t total = 0;
   auto carve = [&total](size_t bytes) { size_t off = total; total += round_up(bytes, 256); return off; };
@@ -155,10 +155,9 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
   const size_t o_regions = carve((size_t)region_bytes);
-  const size_t o_flen = carve((size_t)n_tasks * 4), o_fslow = carve((size_t)n_tasks * 8);
-  const size_t o_fvar = carve((size_t)n_tasks * 4), o_fhdr = carve((size_t)n_tasks * 16);
+  const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve((size_t)n_tasks * 16);
   const size_t o_image = carve((size_t)worst_image), o_hdr = carve(16);
-  const size_t o_counters = carve(24), o_done = carve(4), o_err = carve(4);
+  const size_t o_counters = carve(24), o_rebuild = carve(32), o_err = carve(4);
 
 #define LOAD_TRY(expr)                                                     \
   do {                                                                     \
@@ -198,14 +197,12 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.count_by_id = reinterpret_cast<uint32_t *>(base + o_count);
   d.regions = base + o_regions;
   d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
-  d.f_slow = reinterpret_cast<uint2 *>(base + o_fslow);
-  d.f_var_bytes = reinterpret_cast<uint32_t *>(base + o_fvar);
-  d.f_hdr = reinterpret_cast<uint4 *>(base + o_fhdr);
+  d.slow = reinterpret_cast<uint4 *>(base + o_slow);
   d.image = base + o_image;
   d.image_capacity = (uint32_t)worst_image;
   d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
   d.counters = reinterpret_cast<unsigned long long *>(base + o_counters);
-  d.done_ctr = reinterpret_cast<uint32_t *>(base + o_done);
+  d.rebuild_ctr = reinterpret_cast<uint32_t *>(base + o_rebuild);
   d.err = reinterpret_cast<uint32_t *>(base + o_err);
   c->slot_of_id.swap(slot_of_id);
   c->task_off.swap(task_off);

@@ -18,83 +18,111 @@ namespace infaas {
 //   Pd[0..Ks)  distinct pred_lat values ascending,  Ad[0..Ka)  distinct acc_bp ascending,
 //   r(slo) = #{Pd <= slo},  k(min_acc) = #{Ad < min_acc},
 //   T2[r][k] = first position whose pred_lat is among the r smallest values and whose
-//              acc_bp is not among the k smallest values (0xFF: none) -- the answer.
-// r comes from a table of SLO_BUCKETS records indexed by a monotone bucket of slo (top bits
-// of slo converted to float, shifted by `sh`, relative to `bmin`); a record holds the rank
-// below the bucket and the one distinct value inside it (as a 24-bit offset from the
-// bucket's smallest slo).  A bucket holding two or more values sends the query to two
-// extra rows of T2 that contain only 0xFF, i.e. to the exact slow path.  k comes from a
-// bitmap over acc values with running popcounts (24 bitmap bits + 8 prefix bits per word),
-// exact at one basis point.
+//              acc_bp is not among the k smallest values, or F if there is none.
 //
-// Image (what the selection kernel stages in shared memory), all parts 64-byte aligned:
-//   hdr    uint4[n_tasks + 1]   fast-path parameters (below); entry n_tasks serves queries
-//                               whose task is out of range
-//   slow   uint2[n_tasks + 1]   slow-path parameters: aux offset, F | Ks<<8 | Ka<<16
-//   slo    u32[n_tasks + 1][SLO_BUCKETS]   SLO records: lb << 24 | delta
-//   dummy  64 bytes of 0x00, 64 bytes of 0xFF   (what tasks without an index point at)
-//   var    per-task blocks back to back, each:
-//          ids u32[8*Fp8], Pd u32[8*Fp8], acc bitmap u32[nbw], T2 u8[(Ks+3)*width],
-//          aux (what the nearest-miss search reads, see AuxLayout), padded to 64 bytes
+// r comes from one record of a table of SLO_BUCKETS records per task.  The bucket of an
+// SLO is  j = clamp((bits(slo) >> S) - bmin, 0, 255)  with bits(x) = the IEEE-754 pattern
+// of x converted to float toward zero (a monotone, roughly logarithmic code) and S = 16..23
+// chosen per task.  A record is  R << 24 | C  and  r = (record + (slo & 0xFFFFFF)) >> 24:
+//   - no distinct latency inside the bucket: R = the rank there, C = 0 (never carries);
+//   - one latency `thr` inside it, and all SLOs of the bucket agree in their top byte:
+//     R = rank below, C = 0xFFFFFF - ((thr - 1) & 0xFFFFFF), so the add carries into R
+//     exactly when slo >= thr;
+//   - otherwise R = Ks + 1, C = 0: row Ks + 1 of T2 holds only F, which sends the query to
+//     the exact slow path.
+// k comes from a bitmap over accuracy values with running popcounts (24 bitmap bits and an
+// 8-bit prefix count per word), exact at one basis point.
 //
-// hdr words (offsets are bytes from the start of the image, 18 bits):
-//   x = ids_off | acc_min << 18            y = bitmap_off | width << 18
-//   z = t2_off | sh << 18 | flags << 21    w = bmin | x_max << 15     (x_max = 24*nbw - 1)
+// Image (what the selection kernel stages in shared memory):
+//   hdr    (n_tasks + 1) x 128 bytes: 8 identical copies of a 16-byte header per task, so
+//          that the 8 lanes served by one shared-memory wavefront never collide; entry
+//          n_tasks serves queries whose task is out of range
+//   rec    (n_tasks + 1) x SLO_BUCKETS u32 records
+//   dummy  64 bytes (what tasks without an index point at: every query of theirs reads
+//          "none" and goes to the slow path)
+//   var    per-task blocks, each 64-byte aligned:
+//          ids   u32[F + 1] in REVERSE order: ids[p] sits at t2_off - 4 - 4p, and the slot
+//                of p = F holds PENDING -- the fast path needs no compare for "none"
+//          T2    u8[(Ks + 2) * (Ka + 1)]  at t2_off
+//          bitmap u32[nbw]
+//          slow-path tables (SlowLayout below)
 //
-// Per task in its region (global memory): keys u64[V] (pred_lat | acc_bp << 32, scan
-// order, F used), ids u32[V]; then, 64-byte aligned, the var block before it is packed.
+// Header words:
+//   w0 = float 2^-S          w1 = float -bmin
+//   w2 = t2_off / 4 | (Ka + 1) << 16 | nbw << 24
+//   w3 = acc_lo | cb << 16    acc_lo = multiple of 24 at or below the smallest accuracy,
+//                             cb = bitmap_off / 4 - acc_lo / 24 (word w of the bitmap, for
+//                             an accuracy a clamped to [acc_lo, acc_lo + 24 nbw - 1], is
+//                             word cb + a / 24 of the image)
+//
+// Per task in global memory (`regions`): keys u64[V] (pred_lat | acc_bp << 32, scan order,
+// F used) and ids u32[V], for lists without an index and for inspection.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
 constexpr uint32_t ACC_WORD_BITS = 24;
-constexpr uint32_t MAX_ACC_WORDS = 420;          // covers 0..10000 bp at 24 per word
-constexpr uint32_t IMAGE_OFFSET_LIMIT = 1u << 18;
-constexpr uint32_t HDR_FLAG_INVALID = 1u;        // no variant (or task out of range): answer INVALID
-constexpr uint32_t HDR_FLAG_NOT_INDEXED = 2u;    // list without index: the slow path walks it
+constexpr uint32_t MAX_ACC_WORDS = 255;          // nbw is an 8-bit field: 6120 basis points
+constexpr uint32_t HDR_BYTES = 128;              // 8 copies x 16 bytes
+constexpr uint32_t IMAGE_WORD_LIMIT = 1u << 16;  // t2_off / 4 and cb are 16-bit fields
+constexpr uint32_t SLO_CAP_US = 1u << 26;        // latencies above this share the last bucket
+constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-2)
+
+constexpr uint32_t TASK_FLAG_INVALID = 1u;       // no variant: answer INFAAS_INVALID
+constexpr uint32_t TASK_FLAG_NOT_INDEXED = 2u;   // list without index: the slow path walks it
 
 inline __host__ __device__ uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-inline __host__ __device__ uint32_t image_slow_offset(uint32_t n_tasks) { return round_up_u32(16u * (n_tasks + 1u), 64u); }
-inline __host__ __device__ uint32_t image_slo_offset(uint32_t n_tasks) {
-  return image_slow_offset(n_tasks) + round_up_u32(8u * (n_tasks + 1u), 64u);
-}
+inline __host__ __device__ uint32_t image_rec_offset(uint32_t n_tasks) { return HDR_BYTES * (n_tasks + 1u); }
 inline __host__ __device__ uint32_t image_dummy_offset(uint32_t n_tasks) {
-  return image_slo_offset(n_tasks) + 4u * SLO_BUCKETS * (n_tasks + 1u);
+  return image_rec_offset(n_tasks) + 4u * SLO_BUCKETS * (n_tasks + 1u);
 }
-inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) { return image_dummy_offset(n_tasks) + 128u; }
+inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) { return image_dummy_offset(n_tasks) + 64u; }
 
-// Byte offsets inside the aux part of a var block, for a list of F entries with Ks / Ka
-// distinct latencies / accuracies.
-//   bestA[r], r in 0..Ks: position of the highest accuracy among the r smallest latencies
-//   bestB[k], k in 0..Ka: position of the lowest latency among all but the k smallest accuracies
-//   order[o]: positions sorted by latency rank; ordRank[o]: that rank; ordStart[r]: first o of rank r
-//   idxA[p], idxP[p]: accuracy / latency rank of position p;  Ad u16[Ka]: distinct accuracies
-struct AuxLayout {
-  uint32_t bestA, bestB, order, ordRank, ordStart, idxA, idxP, Ad, bytes;
+// Byte offsets of the slow-path tables inside a task's block, relative to their start
+// (8-byte aligned), for a list of F entries with Ks / Ka distinct latencies / accuracies.
+//   walk[o]   uint2 (pred_lat, acc | position << 16), entries in ascending latency (ties
+//             in position order)
+//   bestB[k]  uint2 (pred_lat, position) of the lowest-latency entry among those whose
+//             accuracy rank is >= k (first position among equals); position 0xFF if none
+//   Pd[i]     u32 distinct latencies
+//   bestA[r]  u32 acc | position << 16 of the highest-accuracy entry among those whose
+//             latency rank is < r (first position among equals); position 0xFF if none
+//   ordStart[r] u8 first walk index whose latency rank is >= r
+struct SlowLayout {
+  uint32_t walk, bestB, Pd, bestA, ordStart, bytes;
 };
-inline __host__ __device__ AuxLayout aux_layout(uint32_t F, uint32_t Ks, uint32_t Ka) {
-  AuxLayout L;
-  L.bestA = 0;
-  L.bestB = L.bestA + Ks + 1u;
-  L.order = L.bestB + Ka + 1u;
-  L.ordRank = L.order + F;
-  L.ordStart = L.ordRank + F;
-  L.idxA = L.ordStart + Ks + 1u;
-  L.idxP = L.idxA + F;
-  L.Ad = (L.idxP + F + 1u) & ~1u;
-  L.bytes = L.Ad + 2u * Ka;
+inline __host__ __device__ SlowLayout slow_layout(uint32_t F, uint32_t Ks, uint32_t Ka) {
+  SlowLayout L;
+  L.walk = 0;
+  L.bestB = L.walk + 8u * F;
+  L.Pd = L.bestB + 8u * (Ka + 1u);
+  L.bestA = L.Pd + 4u * Ks;
+  L.ordStart = L.bestA + 4u * (Ks + 1u);
+  L.bytes = round_up_u32(L.ordStart + Ks + 1u, 8u);
   return L;
 }
 
-// Worst-case bytes of one task's var block and of its region.
-inline __host__ __device__ uint32_t var_capacity(uint32_t V) {
-  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
-  return round_up_u32(8u * round_up_u32(F, 8) + 4u * MAX_ACC_WORDS + (F + 3u) * (F + 2u) +
-                          aux_layout(F, F, F).bytes, 64u);
+// Offsets inside a task's block and its size.
+struct BlockLayout {
+  uint32_t t2, bitmap, slow, bytes;   // ids start at 0; t2 = 4 (F + 1)
+};
+inline __host__ __device__ BlockLayout block_layout(uint32_t F, uint32_t Ks, uint32_t Ka, uint32_t nbw) {
+  BlockLayout B;
+  B.t2 = 4u * (F + 1u);
+  B.bitmap = round_up_u32(B.t2 + (Ks + 2u) * (Ka + 1u), 4u);
+  B.slow = round_up_u32(B.bitmap + 4u * nbw, 8u);
+  B.bytes = round_up_u32(B.slow + slow_layout(F, Ks, Ka).bytes, 64u);
+  return B;
 }
-inline __host__ __device__ uint32_t region_var_offset(uint32_t V) { return round_up_u32(12u * V, 64u); }
-inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return region_var_offset(V) + var_capacity(V); }
+// Worst-case bytes of one task's block.
+inline __host__ __device__ uint32_t block_capacity(uint32_t V) {
+  const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
+  return block_layout(F, F, F, MAX_ACC_WORDS).bytes;
+}
+inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_up_u32(12u * V, 64u); }
 
+// Slow-path parameters of a task (one uint4 per task, global memory).
+//   x = image offset of the slow tables   y = F | Ks << 8 | Ka << 16   z = flags   w = 0
 // ---------------------------------------------------------------------------------------
 // Device catalog.  "Slot" order: variants bucketed by task, ascending id inside a task;
 // task t owns slots task_off[t] .. task_off[t+1]-1 and all s_* arrays are indexed by slot.
@@ -116,18 +144,16 @@ struct DeviceCatalog {
   unsigned long long *s_served;
   uint32_t *count_by_id;     // [n_variants], zero between windows
 
-  unsigned char *regions;    // per task: keys, ids, then the var block before packing
+  unsigned char *regions;    // per task: keys u64[V], ids u32[V] (scan order)
   uint32_t *f_len;           // [n_tasks] list length F
-  uint32_t *f_var_bytes;     // [n_tasks] bytes of the task's var block (0 if not indexed)
-  uint4 *f_hdr;              // [n_tasks] hdr words with offsets relative to the var block
-  uint2 *f_slow;             // [n_tasks] slow words, aux offset relative to the var block
+  uint4 *slow;               // [n_tasks] slow-path parameters
 
   unsigned char *image;      // packed image, image_capacity bytes, 256-byte aligned
   uint32_t image_capacity;
   uint32_t *image_hdr;       // [4]: bytes, longest list, total entries, tasks not indexed
 
   unsigned long long *counters;  // [3] feasible, no-feasible, invalid
-  uint32_t *done_ctr;            // CTA arrival counter of the rebuild kernel
+  uint32_t *rebuild_ctr;         // [4] CTA arrival counter, block cursor, longest, entries (rebuild kernel)
   uint32_t *err;                 // sticky device error word (0 = fine)
 };
 
@@ -135,7 +161,6 @@ struct DeviceCatalog {
 enum : uint32_t {
   DEV_ERR_NONE = 0,
   DEV_ERR_STAGE_TIMEOUT = 1,   // the bulk copy into shared memory did not complete in time
-  DEV_ERR_IMAGE_OVERFLOW = 2,  // packed image exceeds its buffer (cannot happen by sizing)
 };
 
 // Largest dynamic shared memory the selection kernel may be given (227 KB per CTA on

@@ -6,15 +6,15 @@
 // Each task's scan list is sorted by (cost, pred_lat, -acc, id) and pruned to non-dominated
 // variants, so the answer for a feasible query is the FIRST list position that meets both
 // requirements.  Instead of walking the list, a thread ranks the query's SLO among the
-// list's distinct latencies (one bucket record, one comparison) and its minimum accuracy
-// among the list's distinct accuracies (one bitmap word, one popcount) and reads the
-// answer's position from a small per-task table indexed by the two ranks (layout in
-// common.cuh): five shared-memory loads per query, no loop.  The packed image of all
-// tasks is staged in shared memory once per CTA with bulk asynchronous copies (TMA,
-// mbarrier completion); queries stream through with 128-bit loads and stores, four per
-// thread and iteration.  Queries without a feasible variant (and those of a task whose list
-// is too long for the index) are parked in a per-warp list and resolved 32 at a time with
-// all lanes busy.
+// list's distinct latencies (one bucket record, one add) and its minimum accuracy among
+// the list's distinct accuracies (one bitmap word, one popcount) and reads the answer's
+// position from a small per-task table indexed by the two ranks (layout in common.cuh):
+// five shared-memory loads per query, no loop, no compare.  The packed image of all tasks
+// is staged in shared memory once per CTA with bulk asynchronous copies (TMA, mbarrier
+// completion); queries stream through with 128-bit loads and stores, four per thread and
+// iteration.  Queries the tables cannot answer (nothing feasible, an SLO bucket holding
+// several latencies, a task without index) come out of the fast path as PENDING; they are
+// parked per warp in shared memory with their data and resolved 32 at a time.
 #include "common.cuh"
 
 namespace infaas {
@@ -24,27 +24,24 @@ namespace {
 constexpr int SELECT_THREADS = 1024;
 constexpr int SELECT_WARPS = SELECT_THREADS / 32;
 constexpr uint32_t WARP_TILE = 128;              // queries per warp and iteration
-constexpr uint32_t PARK_CAP = 32 + WARP_TILE;    // parked queries per warp
-constexpr uint32_t PARK_BYTES = SELECT_WARPS * PARK_CAP * 4;
+constexpr uint32_t PARK_CAP = 64;                // parked queries per warp (flushed at 32)
+constexpr uint32_t PARK_BYTES = SELECT_WARPS * PARK_CAP * 12;
 constexpr uint32_t STAGE_CHUNK = 32768;          // bytes per bulk copy
 constexpr uint32_t STAGE_POLL_LIMIT = 1u << 22;  // bounded wait on the staging barrier
-constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-3)
+constexpr uint32_t MAX_SPAN = 1u << 31;          // queries per CTA (offsets are 32-bit)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
 
-// Stage `bytes` (multiple of 16) from global `src` (16-byte aligned) into shared `dst`.
-// Returns false if the copy did not complete within the poll limit.
-__device__ __forceinline__ bool stage_image(unsigned char *dst, const unsigned char *src,
-                                            uint32_t bytes, unsigned long long *mbar) {
+// Start staging `bytes` (multiple of 16) from global `src` (16-byte aligned) into shared
+// `dst`; completion is signalled on `mbar`.
+__device__ __forceinline__ void stage_begin(unsigned char *dst, const unsigned char *src, uint32_t bytes,
+                                            unsigned long long *mbar) {
   const uint32_t bar = smem_u32(mbar);
   if (threadIdx.x == 0) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
     for (uint32_t off = 0; off < bytes; off += STAGE_CHUNK) {
@@ -55,6 +52,13 @@ __device__ __forceinline__ bool stage_image(unsigned char *dst, const unsigned c
           : "memory");
     }
   }
+  __syncthreads();   // the barrier is initialised before anyone polls it
+}
+
+// Wait for the staged bytes.  Returns false (all threads) if they did not arrive within
+// the poll limit.
+__device__ __forceinline__ bool stage_wait(unsigned long long *mbar) {
+  const uint32_t bar = smem_u32(mbar);
   uint32_t done = 0;
   for (uint32_t it = 0; it < STAGE_POLL_LIMIT && !done; ++it) {
     asm volatile(
@@ -78,9 +82,6 @@ struct SharedImage {
   __device__ __forceinline__ uint32_t u32(uint32_t off) const {
     uint32_t v; asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
   }
-  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
-    uint32_t v; asm("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(base + off)); return v;
-  }
   __device__ __forceinline__ uint2 v2(uint32_t off) const {
     uint2 v; asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(base + off)); return v;
   }
@@ -97,9 +98,6 @@ struct GlobalImage {
   __device__ __forceinline__ uint32_t u32(uint32_t off) const {
     return __ldg(reinterpret_cast<const uint32_t *>(base + off));
   }
-  __device__ __forceinline__ uint32_t u16(uint32_t off) const {
-    return __ldg(reinterpret_cast<const uint16_t *>(base + off));
-  }
   __device__ __forceinline__ uint2 v2(uint32_t off) const {
     return __ldg(reinterpret_cast<const uint2 *>(base + off));
   }
@@ -108,103 +106,103 @@ struct GlobalImage {
   }
 };
 
-// k = #{distinct list accuracies < min_acc}, from the bitmap with running popcounts.
+// floor(a / 24) for a < 2^16 as the high half of a product (multiply pipe).
+__device__ __forceinline__ uint32_t div24(uint32_t a) { return __umulhi(a, 178956971u); }
+
+// k = #{distinct list accuracies < min_acc} from the bitmap with running popcounts.
+// w2, w3: header words (see common.cuh).
 template <class Img>
-__device__ __forceinline__ uint32_t acc_rank(const Img &img, uint32_t bitmap_off, uint32_t acc_min,
-                                             uint32_t x_max, uint32_t min_acc) {
-  const uint32_t x = min(max(min_acc, acc_min) - acc_min, x_max);
-  const uint32_t w = (x * 43691u) >> 20;                    // x / 24 for x < 2^16
-  const uint32_t word = img.u32(bitmap_off + (w << 2));
-  return (word >> 24) + __popc(word & ((1u << (x - w * ACC_WORD_BITS)) - 1u));
+__device__ __forceinline__ uint32_t acc_rank(const Img &img, uint32_t w2, uint32_t w3, uint32_t min_acc) {
+  const uint32_t acc_lo = w3 & 0xFFFFu, cb = __umulhi(w3, 1u << 16), nbw = __umulhi(w2, 1u << 8);
+  const uint32_t a = min(max(min_acc, acc_lo), acc_lo + ACC_WORD_BITS * nbw - 1u);
+  const uint32_t w = div24(a);
+  const uint32_t word = img.u32((cb + w) << 2);
+  const uint32_t below = word & ((1u << (a - w * ACC_WORD_BITS)) - 1u);   // prefix byte masked off: shift < 24
+  return __umulhi(word, 1u << 8) + __popc(below);
 }
 
-// Fast path, straight-line: five loads.  Returns the decision, INFAAS_INVALID, or PENDING
-// when the query needs the slow path: nothing feasible, an SLO bucket with several values,
-// or a task whose list has no index (those read 0xFF from T2 by construction).
+// Fast path, straight-line: five loads, no compare.  Returns the variant id, or PENDING
+// when the tables cannot answer (nothing feasible, an SLO bucket with several latencies,
+// a task without index or out of range).  `hdr_lane` = 16 * (lane & 7): which of the 8
+// header copies this lane reads.
 template <class Img>
-__device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks, uint32_t slo_off,
-                                                uint32_t task, uint32_t slo, uint32_t min_acc) {
+__device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks, uint32_t rec_off,
+                                                uint32_t hdr_lane, uint32_t task, uint32_t slo,
+                                                uint32_t min_acc) {
   const uint32_t t = min(task, n_tasks);
-  const uint4 h = img.v4(t << 4);
-  const uint32_t sh = (h.z >> 18) & 7u, bmin = h.w & 0x7FFFu;
-  // r = #{distinct list latencies <= slo}: bucket record + one comparison
-  const uint32_t b = (__float_as_uint(__uint2float_rz(slo)) >> 16) >> sh;
-  const uint32_t j = min(max(b, bmin) - bmin, SLO_BUCKETS - 1u);
-  const uint32_t lo = j ? __float2uint_ru(__uint_as_float((bmin + j) << (sh + 16u))) : 0u;
-  const uint32_t rec = img.u32(slo_off + (((t << 8) + j) << 2));
-  const uint32_t r = (rec >> 24) + ((slo - lo) >= (rec & 0x00FFFFFFu));
-  const uint32_t k = acc_rank(img, h.y & 0x3FFFFu, h.x >> 18, h.w >> 15, min_acc);
-  const uint32_t pos = img.u8((h.z & 0x3FFFFu) + r * (h.y >> 18) + k);
-  const bool none = pos == 0xFFu;
-  const uint32_t id = img.u32((h.x & 0x3FFFFu) + (none ? 0u : pos << 2));
-  return none ? (((h.z >> 21) & HDR_FLAG_INVALID) ? INFAAS_INVALID : PENDING) : id;
+  const uint4 h = img.v4(t * HDR_BYTES + hdr_lane);
+  // bucket of the SLO: floor(bits(slo) * 2^-S) - bmin, saturated to 0..255 by the conversion
+  const float code = __uint2float_rz(__float_as_uint(__uint2float_rz(slo)));
+  uint32_t j;
+  asm("cvt.rmi.sat.u8.f32 %0, %1;" : "=r"(j) : "f"(fmaf(code, __uint_as_float(h.x), __uint_as_float(h.y))));
+  const uint32_t rec = img.u32(rec_off + t * (4u * SLO_BUCKETS) + (j << 2));
+  const uint32_t r = __umulhi(rec + (slo & 0x00FFFFFFu), 1u << 8);
+  const uint32_t k = acc_rank(img, h.z, h.w, min_acc);
+  const uint32_t t2 = (h.z & 0xFFFFu) << 2, width = (h.z >> 16) & 0xFFu;
+  const uint32_t pos = img.u8(t2 + r * width + k);
+  return img.u32(t2 - 4u - (pos << 2));
 }
 
-// d = 10^4 * over_lat + slo * under_acc (64-bit).
-__device__ __forceinline__ unsigned long long miss_distance(uint32_t pred, uint32_t acc, uint32_t slo,
-                                                            uint32_t min_acc) {
-  const uint32_t over = pred > slo ? pred - slo : 0u;
-  const uint32_t under = min_acc > acc ? min_acc - acc : 0u;
-  return (unsigned long long)over * 10000ull + (unsigned long long)slo * under;
-}
-
-// Slow path for a parked query (never an invalid one).
-//   Indexed list: exact ranks (binary search over Pd), then T2.  If nothing is feasible the
-//   nearest miss is the entry smallest in (d, position) -- position order is (cost,
-//   pred_lat, -acc, id) order.  Entries that meet the SLO all miss the accuracy, the best
-//   of them is the one with the highest accuracy (bestA); entries that meet the accuracy
-//   all miss the SLO, the best being the one with the lowest latency (bestB); an entry
-//   that misses both can only win with accuracy above bestA's, latency not above bestB's
-//   and a latency overshoot that alone stays below the best distance so far, so the walk
-//   in latency order stops early.
+// Slow path for a parked query.
+//   Indexed list: exact ranks (binary search over the distinct latencies), then T2.  If
+//   nothing is feasible the nearest miss is the entry smallest in (d, position), with
+//   d = 10^4 * max(0, pred - slo) + slo * max(0, min_acc - acc) in 64 bits -- position
+//   order is (cost, pred_lat, -acc, id) order.  Entries that meet the SLO all miss the
+//   accuracy, the best of them is the one with the highest accuracy (bestA); entries that
+//   meet the accuracy all miss the SLO, the best being the one with the lowest latency
+//   (bestB); an entry that misses both can only win with accuracy above bestA's, latency
+//   not above bestB's and a latency overshoot that alone stays below the best distance so
+//   far, so the walk in latency order stops early.
 //   List without index: walk it in global memory, for a feasible entry, then for the distance.
 template <class Img>
 __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t task,
                                                 uint32_t slo, uint32_t min_acc) {
-  const uint4 h = img.v4(task << 4);
+  if (task >= c.n_tasks) return INFAAS_INVALID;
+  const uint4 sl = __ldg(c.slow + task);
+  if (sl.z & TASK_FLAG_INVALID) return INFAAS_INVALID;
   unsigned long long best = ~0ull;
-  uint32_t best_i = 0;
-  if (!((h.z >> 21) & HDR_FLAG_NOT_INDEXED)) {
-    const uint2 sl = img.v2(image_slow_offset(c.n_tasks) + (task << 3));
+  uint32_t best_p = 0;
+  if (!(sl.z & TASK_FLAG_NOT_INDEXED)) {
     const uint32_t F = sl.y & 0xFFu, Ks = (sl.y >> 8) & 0xFFu, Ka = sl.y >> 16;
-    const uint32_t ids_off = h.x & 0x3FFFFu, pd_off = ids_off + (((F + 7u) >> 3) << 5);
-    const AuxLayout AL = aux_layout(F, Ks, Ka);
-    const uint32_t aux = sl.x;
-    uint32_t lo = 0, hi = Ks;                              // r = #{Pd <= slo}
-    while (lo < hi) {
-      const uint32_t mid = (lo + hi) >> 1;
-      if (img.u32(pd_off + (mid << 2)) <= slo) lo = mid + 1; else hi = mid;
+    const SlowLayout SL = slow_layout(F, Ks, Ka);
+    const uint32_t so = sl.x;
+    const uint4 h = img.v4(task * HDR_BYTES);
+    const uint32_t t2 = (h.z & 0xFFFFu) << 2, width = (h.z >> 16) & 0xFFu;
+    uint32_t r = 0;                                            // r = #{Pd <= slo}
+#pragma unroll
+    for (uint32_t step = 128; step; step >>= 1) {
+      const uint32_t probe = r + step;
+      if (probe <= Ks && img.u32(so + SL.Pd + ((probe - 1u) << 2)) <= slo) r = probe;
     }
-    const uint32_t r = lo;
-    const uint32_t k = acc_rank(img, h.y & 0x3FFFFu, h.x >> 18, h.w >> 15, min_acc);
-    const uint32_t pos = img.u8((h.z & 0x3FFFFu) + r * (h.y >> 18) + k);
-    if (pos != 0xFFu) return img.u32(ids_off + (pos << 2));
-    uint32_t acc_rank_floor = 0;          // candidates need accuracy rank >= this
-    uint32_t lat_rank_cap = Ks;           // ... and latency rank < this
+    const uint32_t k = acc_rank(img, h.z, h.w, min_acc);
+    const uint32_t pos = img.u8(t2 + r * width + k);
+    if (pos < F) return img.u32(t2 - 4u - (pos << 2));
+    uint32_t acc_floor = 0;               // candidates that miss both need accuracy >= this
+    uint32_t pred_cap = 0xFFFFFFFFu;      // ... and latency <= this
     if (r > 0) {                          // some entry meets the SLO (and misses the accuracy)
-      const uint32_t pA = img.u8(aux + AL.bestA + r), ia = img.u8(aux + AL.idxA + pA);
-      best = (unsigned long long)slo * (min_acc - img.u16(aux + AL.Ad + (ia << 1)));
-      best_i = pA;
-      acc_rank_floor = ia + 1u;
+      const uint32_t A = img.u32(so + SL.bestA + (r << 2));
+      best = (unsigned long long)slo * (min_acc - (A & 0xFFFFu));
+      best_p = A >> 16;
+      acc_floor = (A & 0xFFFFu) + 1u;
     }
     if (k < Ka) {                         // some entry meets the accuracy (and misses the SLO)
-      const uint32_t pB = img.u8(aux + AL.bestB + k), ip = img.u8(aux + AL.idxP + pB);
-      const unsigned long long d = (unsigned long long)(img.u32(pd_off + (ip << 2)) - slo) * 10000ull;
-      if (d < best || (d == best && pB < best_i)) { best = d; best_i = pB; }
-      lat_rank_cap = ip + 1u;
+      const uint2 Bv = img.v2(so + SL.bestB + (k << 3));
+      const unsigned long long d = (unsigned long long)(Bv.x - slo) * 10000ull;
+      if (d < best || (d == best && Bv.y < best_p)) { best = d; best_p = Bv.y; }
+      pred_cap = Bv.x;
     }
-    for (uint32_t o = img.u8(aux + AL.ordStart + r); o < F; ++o) {   // latency ranks >= r
-      const uint32_t ip = img.u8(aux + AL.ordRank + o);
-      if (ip >= lat_rank_cap) break;
-      const unsigned long long over = (unsigned long long)(img.u32(pd_off + (ip << 2)) - slo) * 10000ull;
+    for (uint32_t o = img.u8(so + SL.ordStart + r); o < F; ++o) {   // latencies above the SLO, ascending
+      const uint2 e = img.v2(so + SL.walk + (o << 3));
+      if (e.x > pred_cap) break;
+      const unsigned long long over = (unsigned long long)(e.x - slo) * 10000ull;
       if (over > best) break;             // later entries overshoot the SLO even more
-      const uint32_t p = img.u8(aux + AL.order + o), ia = img.u8(aux + AL.idxA + p);
-      if (ia >= acc_rank_floor && ia < k) {
-        const unsigned long long d = over + (unsigned long long)slo * (min_acc - img.u16(aux + AL.Ad + (ia << 1)));
-        if (d < best || (d == best && p < best_i)) { best = d; best_i = p; }
+      const uint32_t acc = e.y & 0xFFFFu, p = e.y >> 16;
+      if (acc >= acc_floor && acc < min_acc) {
+        const unsigned long long d = over + (unsigned long long)slo * (min_acc - acc);
+        if (d < best || (d == best && p < best_p)) { best = d; best_p = p; }
       }
     }
-    return INFAAS_NO_FEASIBLE | img.u32(ids_off + (best_i << 2));
+    return INFAAS_NO_FEASIBLE | img.u32(t2 - 4u - (best_p << 2));
   }
   const uint32_t F = __ldg(c.f_len + task);
   const uint32_t V = __ldg(c.task_off + task + 1) - __ldg(c.task_off + task);
@@ -217,10 +215,12 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
   }
   for (uint32_t i = 0; i < F; ++i) {
     const unsigned long long e = __ldg(keys + i);
-    const unsigned long long d = miss_distance((uint32_t)e, (uint32_t)(e >> 32), slo, min_acc);
-    if (d < best) { best = d; best_i = i; }
+    const uint32_t pred = (uint32_t)e, acc = (uint32_t)(e >> 32);
+    const unsigned long long d = (unsigned long long)(pred > slo ? pred - slo : 0u) * 10000ull +
+                                 (unsigned long long)slo * (min_acc > acc ? min_acc - acc : 0u);
+    if (d < best) { best = d; best_p = i; }
   }
-  return INFAAS_NO_FEASIBLE | __ldg(ids + best_i);
+  return INFAAS_NO_FEASIBLE | __ldg(ids + best_p);
 }
 
 struct Queries {
@@ -230,109 +230,119 @@ struct Queries {
   uint32_t *__restrict__ decision;
 };
 
-// Resolve up to 32 parked queries, one per lane.  `rel` is the query's offset from `q0`.
+// A warp's park list in shared memory: offset of the query from the CTA's first query,
+// task | min_acc << 16, and SLO.
+struct Park {
+  uint32_t *rel, *ta, *slo;
+  uint32_t cnt;
+};
+
+// Resolve the 32 parked queries [first, first + count), one per lane.
 template <class Img>
-__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, const Queries &q,
-                                               uint64_t q0, const uint32_t *park, uint32_t first,
-                                               uint32_t count) {
+__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, uint32_t *out,
+                                               const Park &pk, uint32_t first, uint32_t count) {
   const uint32_t lane = threadIdx.x & 31;
   if (lane < count) {
-    const uint64_t i = q0 + park[first + lane];
-    q.decision[i] = decide_slow(img, c, q.task[i], q.slo[i], q.min_acc[i]);
+    const uint32_t ta = pk.ta[first + lane];
+    out[pk.rel[first + lane]] = decide_slow(img, c, ta & 0xFFFFu, pk.slo[first + lane], ta >> 16);
   }
 }
 
-// Append the lanes with `pending` to the warp's park list (all lanes call this).
-__device__ __forceinline__ void park_append(uint32_t *park, uint32_t &cnt, bool pending, uint32_t rel) {
-  const unsigned m = __ballot_sync(0xFFFFFFFFu, pending);
-  if (pending) park[cnt + __popc(m & ((1u << (threadIdx.x & 31)) - 1u))] = rel;
-  cnt += __popc(m);
+// Park the queries a lane holds whose bit is set in `pm` (bit i = i-th of its four
+// queries, data in ta[i] / s[i], offset rel + i); flush whenever 32 are waiting.  All
+// lanes of the warp call this together.
+template <class Img>
+__device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatalog &c, uint32_t *out, Park &pk,
+                                               uint32_t pm, uint32_t rel, const uint32_t (&ta)[4],
+                                               const uint32_t (&s)[4]) {
+  const uint32_t lane_lt = (1u << (threadIdx.x & 31)) - 1u;
+  unsigned m;
+  while ((m = __ballot_sync(0xFFFFFFFFu, pm != 0u)) != 0u) {
+    if (pm) {
+      const uint32_t i = __ffs(pm) - 1u, slot = pk.cnt + __popc(m & lane_lt);
+      pk.rel[slot] = rel + i;
+      pk.ta[slot] = i == 0 ? ta[0] : i == 1 ? ta[1] : i == 2 ? ta[2] : ta[3];
+      pk.slo[slot] = i == 0 ? s[0] : i == 1 ? s[1] : i == 2 ? s[2] : s[3];
+      pm &= pm - 1u;
+    }
+    pk.cnt += __popc(m);
+    __syncwarp();
+    if (pk.cnt >= 32) {
+      pk.cnt -= 32;
+      resolve_parked(img, c, out, pk, pk.cnt, 32);
+      __syncwarp();
+    }
+  }
 }
 
 template <class Img>
 __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
-                                            uint64_t n, uint64_t per_cta, uint32_t *park_all) {
+                                            uint64_t q0, uint32_t span, uint32_t *park_all, uint2 t4, uint4 s4,
+                                            uint2 a4) {
   const uint32_t n_tasks = c.n_tasks;
-  const uint32_t slo_off = image_slo_offset(n_tasks);
+  const uint32_t rec_off = image_rec_offset(n_tasks);
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  uint32_t *park = park_all + warp * PARK_CAP;
-  uint32_t parked = 0;
-  const uint64_t q0 = (uint64_t)blockIdx.x * per_cta;
-  const uint64_t q1 = min(n, q0 + per_cta);
-  if (q0 >= q1) return;
-  const uint64_t span = q1 - q0;                       // < 2^32 (checked by the launcher)
-  const uint64_t full_tiles = span / WARP_TILE;
+  const uint32_t hdr_lane = (lane & 7u) << 4;
+  Park pk;
+  pk.rel = park_all + warp * (3 * PARK_CAP);
+  pk.ta = pk.rel + PARK_CAP;
+  pk.slo = pk.ta + PARK_CAP;
+  pk.cnt = 0;
+  uint32_t *out = q.decision + q0;
+  const uint32_t full_tiles = span / WARP_TILE;
 
-  // full tiles: 4 consecutive queries per lane, 128-bit loads, next tile prefetched
-  uint64_t tile = warp;
-  uint2 t4 = make_uint2(0, 0), a4 = make_uint2(0, 0);
-  uint4 s4 = make_uint4(0, 0, 0, 0);
-  if (tile < full_tiles) {
-    const uint64_t i4 = (q0 + tile * WARP_TILE) / 4 + lane;
-    t4 = __ldcs(reinterpret_cast<const uint2 *>(q.task) + i4);
-    s4 = __ldcs(reinterpret_cast<const uint4 *>(q.slo) + i4);
-    a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
-  }
-  for (; tile < full_tiles; tile += SELECT_WARPS) {
+  // full tiles: 4 consecutive queries per lane, 128-bit loads, next tile prefetched (the
+  // first tile was loaded by the caller while the image was being staged)
+  for (uint32_t tile = warp; tile < full_tiles; tile += SELECT_WARPS) {
     const uint2 t = t4, a = a4;
     const uint4 s = s4;
-    const uint64_t next = tile + SELECT_WARPS;
+    const uint32_t next = tile + SELECT_WARPS;
     if (next < full_tiles) {
-      const uint64_t i4 = (q0 + next * WARP_TILE) / 4 + lane;
+      const uint64_t i4 = (q0 + (uint64_t)next * WARP_TILE) / 4 + lane;
       t4 = __ldcs(reinterpret_cast<const uint2 *>(q.task) + i4);
       s4 = __ldcs(reinterpret_cast<const uint4 *>(q.slo) + i4);
       a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
     }
+    const uint32_t tq[4] = {t.x & 0xFFFFu, t.x >> 16, t.y & 0xFFFFu, t.y >> 16};
+    const uint32_t aq[4] = {a.x & 0xFFFFu, a.x >> 16, a.y & 0xFFFFu, a.y >> 16};
+    const uint32_t sq[4] = {s.x, s.y, s.z, s.w};
     uint4 d;
-    d.x = decide_fast(img, n_tasks, slo_off, t.x & 0xFFFFu, s.x, a.x & 0xFFFFu);
-    d.y = decide_fast(img, n_tasks, slo_off, t.x >> 16, s.y, a.x >> 16);
-    d.z = decide_fast(img, n_tasks, slo_off, t.y & 0xFFFFu, s.z, a.y & 0xFFFFu);
-    d.w = decide_fast(img, n_tasks, slo_off, t.y >> 16, s.w, a.y >> 16);
-    const uint32_t rel = (uint32_t)(tile * WARP_TILE) + lane * 4u;
-    uint32_t *out = q.decision + q0 + rel;
-    const bool any_pending = d.x == PENDING || d.y == PENDING || d.z == PENDING || d.w == PENDING;
-    if (!any_pending) {
-      __stcs(reinterpret_cast<uint4 *>(out), d);
-    } else {            // a parked slot is written later by another lane: leave it alone now
-      if (d.x != PENDING) out[0] = d.x;
-      if (d.y != PENDING) out[1] = d.y;
-      if (d.z != PENDING) out[2] = d.z;
-      if (d.w != PENDING) out[3] = d.w;
-    }
-    if (__any_sync(0xFFFFFFFFu, any_pending)) {
-      park_append(park, parked, d.x == PENDING, rel);
-      park_append(park, parked, d.y == PENDING, rel + 1);
-      park_append(park, parked, d.z == PENDING, rel + 2);
-      park_append(park, parked, d.w == PENDING, rel + 3);
+    d.x = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[0], sq[0], aq[0]);
+    d.y = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[1], sq[1], aq[1]);
+    d.z = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[2], sq[2], aq[2]);
+    d.w = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[3], sq[3], aq[3]);
+    const uint32_t rel = tile * WARP_TILE + lane * 4u;
+    // PENDING slots are overwritten by the lane that resolves them, after a warp barrier
+    __stcs(reinterpret_cast<uint4 *>(out + rel), d);
+    // valid ids stay below 2^31, PENDING has bit 31 set
+    if (__any_sync(0xFFFFFFFFu, (int)(d.x | d.y | d.z | d.w) < 0)) {
+      const uint32_t pm = (d.x >> 31) | ((d.y >> 31) << 1) | ((d.z >> 31) << 2) | ((d.w >> 31) << 3);
+      const uint32_t ta[4] = {tq[0] | (aq[0] << 16), tq[1] | (aq[1] << 16), tq[2] | (aq[2] << 16),
+                              tq[3] | (aq[3] << 16)};
       __syncwarp();
-      while (parked >= 32) {
-        parked -= 32;
-        resolve_parked(img, c, q, q0, park, parked, 32);
-      }
-      __syncwarp();
+      park_and_flush(img, c, out, pk, pm, rel, ta, sq);
     }
   }
   // ragged tail of the CTA's range (fewer than WARP_TILE queries): one warp, scalar accesses
-  const uint64_t tail0 = full_tiles * WARP_TILE;
-  if (tail0 < span && warp == (uint32_t)(full_tiles % SELECT_WARPS)) {
+  const uint32_t tail0 = full_tiles * WARP_TILE;
+  if (tail0 < span && warp == full_tiles % SELECT_WARPS) {
     for (uint32_t j = 0; j < WARP_TILE / 32; ++j) {
-      const uint64_t rel = tail0 + j * 32u + lane;
-      uint32_t d = 0;
+      const uint32_t rel = tail0 + j * 32u + lane;
+      uint32_t d = 0, ta[4] = {0, 0, 0, 0}, sq[4] = {0, 0, 0, 0};
       if (rel < span) {
         const uint64_t i = q0 + rel;
-        d = decide_fast(img, n_tasks, slo_off, q.task[i], q.slo[i], q.min_acc[i]);
-        if (d != PENDING) q.decision[i] = d;
+        const uint32_t tk = q.task[i], ac = q.min_acc[i];
+        sq[0] = q.slo[i];
+        ta[0] = tk | (ac << 16);
+        d = decide_fast(img, n_tasks, rec_off, hdr_lane, tk, sq[0], ac);
+        out[rel] = d;
       }
-      park_append(park, parked, rel < span && d == PENDING, (uint32_t)rel);
-    }
-    __syncwarp();
-    while (parked >= 32) {
-      parked -= 32;
-      resolve_parked(img, c, q, q0, park, parked, 32);
+      __syncwarp();
+      park_and_flush(img, c, out, pk, d >> 31, rel, ta, sq);
     }
   }
   __syncwarp();
-  resolve_parked(img, c, q, q0, park, 0, parked);
+  resolve_parked(img, c, out, pk, 0, pk.cnt);
 }
 
 __global__ void __launch_bounds__(SELECT_THREADS, 1)
@@ -341,18 +351,33 @@ select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint6
   __shared__ __align__(8) unsigned long long mbar;
   uint32_t *park = reinterpret_cast<uint32_t *>(smem);
   unsigned char *staged = smem + PARK_BYTES;
+  const uint64_t q0 = (uint64_t)blockIdx.x * per_cta;
+  if (q0 >= n) return;
+  const uint32_t span = (uint32_t)min(n - q0, per_cta);     // <= MAX_SPAN (checked by the launcher)
   const uint32_t bytes = c.image_hdr[0];
-  if (bytes <= image_smem) {
-    if (!stage_image(staged, c.image, bytes, &mbar)) {
+  const bool in_smem = bytes <= image_smem;
+  if (in_smem) stage_begin(staged, c.image, bytes, &mbar);
+  // first tile of every warp: in flight while the image arrives
+  uint2 t4 = make_uint2(0, 0), a4 = make_uint2(0, 0);
+  uint4 s4 = make_uint4(0, 0, 0, 0);
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp < span / WARP_TILE) {
+    const uint64_t i4 = (q0 + (uint64_t)warp * WARP_TILE) / 4 + lane;
+    t4 = __ldcs(reinterpret_cast<const uint2 *>(q.task) + i4);
+    s4 = __ldcs(reinterpret_cast<const uint4 *>(q.slo) + i4);
+    a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
+  }
+  if (in_smem) {
+    if (!stage_wait(&mbar)) {
       if (threadIdx.x == 0) atomicMax(c.err, (uint32_t)DEV_ERR_STAGE_TIMEOUT);
       return;
     }
     SharedImage img{smem_u32(staged)};
-    select_body(img, c, q, n, per_cta, park);
+    select_body(img, c, q, q0, span, park, t4, s4, a4);
   } else {
     // the image does not fit in shared memory: read it from global memory (L1/L2 resident)
     GlobalImage img{c.image};
-    select_body(img, c, q, n, per_cta, park);
+    select_body(img, c, q, q0, span, park, t4, s4, a4);
   }
 }
 
@@ -374,12 +399,13 @@ cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const 
   if (n == 0) return cudaSuccess;
   image_smem = select_image_smem(image_smem);
   // one CTA per SM; every CTA takes one contiguous range, a multiple of the warp tile
-  uint64_t grid = (uint64_t)sm_count;
   const uint64_t tiles = (n + WARP_TILE - 1) / WARP_TILE;
+  uint64_t grid = (uint64_t)sm_count;
   if (grid > tiles) grid = tiles;
-  const uint64_t per_cta = (tiles + grid - 1) / grid * WARP_TILE;
-  if (per_cta > 0xFFFFFFFFull) return cudaErrorInvalidValue;
+  uint64_t per_cta = (tiles + grid - 1) / grid * WARP_TILE;
+  if (per_cta > MAX_SPAN) per_cta = MAX_SPAN;               // very large batches: more CTAs than SMs
   grid = (n + per_cta - 1) / per_cta;
+  if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
   Queries q{d_task, d_slo, d_min_acc, d_decision};
   select_kernel<<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n,
                                                                                      per_cta);

@@ -143,30 +143,38 @@ __device__ __forceinline__ uint32_t block_excl_scan_flag(bool flag, uint32_t *wa
   return before + in_warp;
 }
 
-// Top 15 bits of a u32 converted to float toward zero: a monotone, roughly logarithmic
-// code (8 exponent bits, 7 mantissa bits).  The selection kernel computes the same code.
-__device__ __forceinline__ uint32_t float_code(uint32_t x) {
-  return __float_as_uint(__uint2float_rz(x)) >> 16;
+// IEEE-754 pattern of a u32 converted to float toward zero: a monotone, roughly logarithmic
+// code.  The selection kernel derives the same bucket from it.
+__device__ __forceinline__ uint32_t float_bits(uint32_t x) { return __float_as_uint(__uint2float_rz(x)); }
+// Smallest u32 whose float_bits is >= pattern (pattern below that of 2^32).
+__device__ __forceinline__ uint32_t float_bits_floor(uint32_t pattern) {
+  return __float2uint_ru(__uint_as_float(pattern));
 }
-// Smallest u32 whose float_code is >= code (code > 0).
-__device__ __forceinline__ uint32_t float_code_floor(uint32_t code) {
-  return __float2uint_ru(__uint_as_float(code << 16));
-}
+constexpr uint32_t BITS_OF_2_POW_32 = 0x4F800000u;
 
 struct IndexScratch {          // shared memory used while building one task's index
-  uint32_t pred[256], Pd[256];
+  uint32_t pred[256], Pd[256], ids[256];
   uint16_t acc[256], Ad[256];
   unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256];
-  uint32_t ks, ka;
+  uint32_t ks, ka, base;
 };
 
-// Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh).
-// S.pred / S.acc hold the list in scan order.  Writes the SLO records straight into the
-// image, the var block into the task's region, and the task's header words (offsets
-// relative to the var block) and var-block size into the per-task arrays.
-__device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint32_t V, IndexScratch &S) {
+// Header of a task without index (also entry n_tasks): every query reads "none".
+__device__ __forceinline__ uint4 dummy_header(uint32_t n_tasks) {
+  const uint32_t dummy = image_dummy_offset(n_tasks);
+  return make_uint4(0u, 0u, ((dummy + 4u) >> 2) | (0u << 16) | (1u << 24), 0u | (((dummy + 8u) >> 2) << 16));
+}
+__device__ __forceinline__ void write_header(const DeviceCatalog &c, uint32_t t, uint4 h) {
+  if (threadIdx.x < HDR_BYTES / 16u) reinterpret_cast<uint4 *>(c.image + HDR_BYTES * t)[threadIdx.x] = h;
+}
+
+// Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh) into
+// a block of the image obtained from the block cursor.  S.pred / S.acc / S.ids hold the
+// list in scan order.  Returns false (all threads) if the list cannot be indexed: its
+// accuracies span more than the bitmap supports, or the block lies beyond what the 16-bit
+// offsets address.
+__device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, IndexScratch &S) {
   const uint32_t tid = threadIdx.x, B = blockDim.x;
-  unsigned char *region = c.regions + c.reg_off[t];
   // distinct values and their ranks
   for (uint32_t p = tid; p < F; p += B) {
     bool fp = true, fa = true;
@@ -200,90 +208,35 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
     for (uint32_t q = 0; q < F; ++q) o += S.idxP[q] < S.idxP[p] || (S.idxP[q] == S.idxP[p] && q < p);
     S.order[o] = (unsigned char)p;
   }
-  __syncthreads();
 
-  // var block layout
-  const uint32_t Fp8 = (F + 7u) / 8u;
-  const uint32_t acc_min = S.Ad[0] & ~3u;
-  const uint32_t nbw = (S.Ad[Ka - 1] - acc_min + 2u + ACC_WORD_BITS - 1u) / ACC_WORD_BITS;
+  // block layout and its place in the image
+  const uint32_t acc_lo = (S.Ad[0] / ACC_WORD_BITS) * ACC_WORD_BITS;
+  const uint32_t nbw = (S.Ad[Ka - 1] + 1u - acc_lo) / ACC_WORD_BITS + 1u;
   const uint32_t width = Ka + 1u;
-  const uint32_t off_pd = 32u * Fp8, off_bitmap = 64u * Fp8, off_t2 = off_bitmap + 4u * nbw;
-  const uint32_t off_aux = (off_t2 + (Ks + 3u) * width + 3u) & ~3u;
-  const AuxLayout AL = aux_layout(F, Ks, Ka);
-  unsigned char *var = region + region_var_offset(V);
-  unsigned char *aux = var + off_aux;
+  const BlockLayout BL = block_layout(F, Ks, Ka, nbw);
+  const SlowLayout SL = slow_layout(F, Ks, Ka);
+  if (tid == 0) {
+    uint32_t base = 0xFFFFFFFFu;
+    if (nbw <= MAX_ACC_WORDS) {
+      base = image_var_offset(c.n_tasks) + atomicAdd(&c.rebuild_ctr[1], BL.bytes);
+      if (base + BL.bytes > c.image_capacity || ((base + BL.bitmap) >> 2) >= IMAGE_WORD_LIMIT) base = 0xFFFFFFFFu;
+    }
+    S.base = base;
+  }
+  __syncthreads();
+  const uint32_t base = S.base;
+  if (base == 0xFFFFFFFFu) return false;
+  unsigned char *blk = c.image + base;
 
-  uint32_t *Pd_hot = reinterpret_cast<uint32_t *>(var + off_pd);
-  for (uint32_t i = tid; i < Ks; i += B) Pd_hot[i] = S.Pd[i];
-  uint16_t *Ad_hot = reinterpret_cast<uint16_t *>(aux + AL.Ad);
-  for (uint32_t i = tid; i < Ka; i += B) Ad_hot[i] = S.Ad[i];
-  // what the nearest-miss search reads
-  for (uint32_t p = tid; p < F; p += B) {
-    aux[AL.order + p] = S.order[p];
-    aux[AL.ordRank + p] = S.idxP[S.order[p]];
-    aux[AL.idxA + p] = S.idxA[p];
-    aux[AL.idxP + p] = S.idxP[p];
-  }
-  for (uint32_t r = tid; r <= Ks; r += B) {
-    uint32_t best = 0xFFu, best_acc = 0, cnt = 0;           // highest accuracy among ranks < r
-    for (uint32_t p = 0; p < F; ++p) {
-      if (S.idxP[p] < r) {
-        ++cnt;
-        if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
-      }
-    }
-    aux[AL.bestA + r] = (unsigned char)best;
-    aux[AL.ordStart + r] = (unsigned char)cnt;
-  }
-  for (uint32_t k = tid; k <= Ka; k += B) {
-    uint32_t best = 0xFFu, best_pred = 0;                    // lowest latency among accuracy ranks >= k
-    for (uint32_t p = 0; p < F; ++p) {
-      if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
-    }
-    aux[AL.bestB + k] = (unsigned char)best;
-  }
+  // ids, reversed; the slot of "position F" holds PENDING
+  uint32_t *ids_end = reinterpret_cast<uint32_t *>(blk + BL.t2);
+  for (uint32_t p = tid; p <= F; p += B) ids_end[-1 - (int)p] = p < F ? S.ids[p] : PENDING;
 
-  // SLO records.  A bucket with two or more values points at row Ks + 1 of T2 (rows Ks + 1
-  // and Ks + 2 hold only 0xFF), so such a query goes to the slow path.
-  const uint32_t cmin = float_code(S.Pd[0]), cmax = float_code(S.Pd[Ks - 1]);
-  uint32_t sh = 0;
-  while ((cmax >> sh) - (cmin >> sh) > SLO_BUCKETS - 1) ++sh;
-  const uint32_t bmin = cmin >> sh;
-  uint32_t *slo_rec = reinterpret_cast<uint32_t *>(c.image + image_slo_offset(c.n_tasks)) + t * SLO_BUCKETS;
-  for (uint32_t j = tid; j < SLO_BUCKETS; j += B) {
-    uint32_t lb = 0, cnt = 0, thr = 0;
-    for (uint32_t i = 0; i < Ks; ++i) {
-      const uint32_t b = min(max(float_code(S.Pd[i]) >> sh, bmin) - bmin, SLO_BUCKETS - 1);
-      lb += b < j;
-      if (b == j) { ++cnt; thr = S.Pd[i]; }
-    }
-    uint32_t rec = (Ks + 1u) << 24;                           // two or more values: slow path
-    if (cnt == 0) {
-      rec = lb ? ((lb - 1u) << 24) : 0x00FFFFFFu;             // always one more than lb - 1 (lb = 0 cannot occur)
-    } else if (cnt == 1) {
-      const uint32_t lo = j ? float_code_floor((bmin + j) << sh) : 0u;
-      const uint32_t delta = thr - lo;
-      if (delta < 0x01000000u) rec = (lb << 24) | delta;
-    }
-    slo_rec[j] = rec;
-  }
-
-  // accuracy bitmap
-  uint32_t *bitmap = reinterpret_cast<uint32_t *>(var + off_bitmap);
-  for (uint32_t w = tid; w < nbw; w += B) {
-    uint32_t bits = 0, prefix = 0;
-    for (uint32_t i = 0; i < Ka; ++i) {
-      const uint32_t x = S.Ad[i] - acc_min, xw = x / ACC_WORD_BITS;
-      prefix += xw < w;
-      if (xw == w) bits |= 1u << (x - xw * ACC_WORD_BITS);
-    }
-    bitmap[w] = (prefix << 24) | bits;
-  }
   // T2, one thread per accuracy rank k: walk the positions in latency-rank order
-  unsigned char *T2 = var + off_t2;
+  unsigned char *T2 = blk + BL.t2;
   for (uint32_t k = tid; k < width; k += B) {
-    uint32_t cur = 0xFFu, o = 0;
-    T2[k] = 0xFFu;                                             // r = 0: no latency is met
+    uint32_t cur = F, o = 0;
+    T2[k] = (unsigned char)F;                                  // r = 0: no latency is met
     for (uint32_t r = 1; r <= Ks; ++r) {
       while (o < F && S.idxP[S.order[o]] == r - 1) {
         const uint32_t p = S.order[o];
@@ -292,15 +245,83 @@ __device__ void build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, uint
       }
       T2[r * width + k] = (unsigned char)cur;
     }
-    T2[(Ks + 1u) * width + k] = 0xFFu;
-    T2[(Ks + 2u) * width + k] = 0xFFu;
+    T2[(Ks + 1u) * width + k] = (unsigned char)F;
   }
-  if (tid == 0) {
-    c.f_hdr[t] = make_uint4(0u | (acc_min << 18), off_bitmap | (width << 18), off_t2 | (sh << 18),
-                            bmin | ((ACC_WORD_BITS * nbw - 1u) << 15));
-    c.f_slow[t] = make_uint2(off_aux, F | (Ks << 8) | (Ka << 16));
-    c.f_var_bytes[t] = round_up_u32(off_aux + AL.bytes, 64u);
+
+  // accuracy bitmap with running popcounts
+  uint32_t *bitmap = reinterpret_cast<uint32_t *>(blk + BL.bitmap);
+  for (uint32_t w = tid; w < nbw; w += B) {
+    uint32_t bits = 0, prefix = 0;
+    for (uint32_t i = 0; i < Ka; ++i) {
+      const uint32_t x = S.Ad[i] - acc_lo, xw = x / ACC_WORD_BITS;
+      prefix += xw < w;
+      if (xw == w) bits |= 1u << (x - xw * ACC_WORD_BITS);
+    }
+    bitmap[w] = (prefix << 24) | bits;
   }
+
+  // what the nearest-miss search reads
+  unsigned char *slow = blk + BL.slow;
+  uint2 *walk = reinterpret_cast<uint2 *>(slow + SL.walk);
+  for (uint32_t o = tid; o < F; o += B) {
+    const uint32_t p = S.order[o];
+    walk[o] = make_uint2(S.pred[p], (uint32_t)S.acc[p] | (p << 16));
+  }
+  uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
+  for (uint32_t i = tid; i < Ks; i += B) Pd_g[i] = S.Pd[i];
+  uint32_t *bestA = reinterpret_cast<uint32_t *>(slow + SL.bestA);
+  for (uint32_t r = tid; r <= Ks; r += B) {
+    uint32_t best = 0xFFu, best_acc = 0, cnt = 0;               // highest accuracy among ranks < r
+    for (uint32_t p = 0; p < F; ++p) {
+      if (S.idxP[p] < r) {
+        ++cnt;
+        if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
+      }
+    }
+    bestA[r] = best_acc | (best << 16);
+    slow[SL.ordStart + r] = (unsigned char)cnt;
+  }
+  uint2 *bestB = reinterpret_cast<uint2 *>(slow + SL.bestB);
+  for (uint32_t k = tid; k <= Ka; k += B) {
+    uint32_t best = 0xFFu, best_pred = 0;                        // lowest latency among accuracy ranks >= k
+    for (uint32_t p = 0; p < F; ++p) {
+      if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
+    }
+    bestB[k] = make_uint2(best_pred, best);
+  }
+
+  // SLO records.  The buckets cover the list's latencies up to SLO_CAP_US; larger ones
+  // share bucket 255.
+  const uint32_t clo = float_bits(S.Pd[0]) >> 16;
+  const uint32_t chi = max(clo, float_bits(min(S.Pd[Ks - 1], SLO_CAP_US)) >> 16);
+  uint32_t sh = 0;
+  while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
+  const uint32_t bmin = clo >> sh, Sh = 16u + sh;
+  uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
+  for (uint32_t j = tid; j < SLO_BUCKETS; j += B) {
+    uint32_t lb = 0, cnt = 0, thr = 0;
+    for (uint32_t i = 0; i < Ks; ++i) {
+      const uint32_t b = min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1);
+      lb += b < j;
+      if (b == j) { ++cnt; thr = S.Pd[i]; }
+    }
+    const uint32_t lo = j ? float_bits_floor((bmin + j) << Sh) : 0u;
+    const uint32_t next = (bmin + j + 1u) << Sh;
+    const uint32_t hi = (j == SLO_BUCKETS - 1 || next >= BITS_OF_2_POW_32) ? 0xFFFFFFFFu : float_bits_floor(next) - 1u;
+    uint32_t r = (Ks + 1u) << 24;                                // exact slow path
+    if (cnt == 0) {
+      r = lb << 24;
+    } else if (cnt == 1 && (lo >> 24) == (hi >> 24)) {
+      r = thr <= lo ? (lb + 1u) << 24 : (lb << 24) | (0x00FFFFFFu - ((thr - 1u) & 0x00FFFFFFu));
+    }
+    rec[j] = r;
+  }
+
+  const uint32_t cb = ((base + BL.bitmap) >> 2) - acc_lo / ACC_WORD_BITS;
+  write_header(c, t, make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
+                                ((base + BL.t2) >> 2) | (width << 16) | (nbw << 24), acc_lo | (cb << 16)));
+  if (tid == 0) c.slow[t] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, 0u);
+  return true;
 }
 
 __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us) {
@@ -395,13 +416,12 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   if ((tid & 31) == 0 && my_kept) atomicAdd(&s_total, my_kept);
   __syncthreads();
   const uint32_t F = s_total;
-  const bool indexed = F > 0 && F <= INDEX_MAX_F;
+  bool indexed = F > 0 && F <= INDEX_MAX_F;
   unsigned char *region = c.regions + c.reg_off[t];
 
-  // 4. compact into the task's region (scan order): keys and ids, and the var block's ids
+  // 4. compact into the task's region (scan order): keys and ids
   unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(region);
   uint32_t *ids_g = reinterpret_cast<uint32_t *>(region + 8u * V);
-  uint32_t *var_ids = reinterpret_cast<uint32_t *>(region + region_var_offset(V));
   uint32_t kept_so_far = 0;
   for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
     const uint32_t p = p0 + tid;
@@ -413,153 +433,50 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
       const uint32_t id = c.s_id[base + (k32[p] & 0xFFFFu)];
       keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
       ids_g[pos] = id;
-      if (indexed) { var_ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }
+      if (indexed) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }
     }
     kept_so_far += total;
   }
   __syncthreads();
-  if (indexed) {
-    build_index(c, t, F, V, S);
-  } else if (tid == 0) {
-    c.f_var_bytes[t] = 0;
+  if (indexed) indexed = build_index(c, t, F, S);
+  if (!indexed) {
+    // no index: header and records that make every query of this task read "none"
+    write_header(c, t, dummy_header(c.n_tasks));
+    uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
+    for (uint32_t j = tid; j < SLO_BUCKETS; j += B) rec[j] = 0u;
+    if (tid == 0) c.slow[t] = make_uint4(0u, 0u, F == 0 ? TASK_FLAG_INVALID : TASK_FLAG_NOT_INDEXED, 0u);
   }
-  if (tid == 0) c.f_len[t] = F;
+  if (t == 0) {
+    // entry n_tasks (queries whose task is out of range) and the dummy block
+    const uint32_t T = c.n_tasks, dummy = image_dummy_offset(T);
+    write_header(c, T, dummy_header(T));
+    uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T)) + T * SLO_BUCKETS;
+    for (uint32_t j = tid; j < SLO_BUCKETS; j += B) rec[j] = 0u;
+    if (tid < 16) reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid == 0 ? PENDING : 0u;
+  }
+  if (tid == 0) {
+    c.f_len[t] = F;
+    atomicMax(&c.rebuild_ctr[2], F);
+    atomicAdd(&c.rebuild_ctr[3], F);
+    if (F > 0 && !indexed) atomicAdd(&c.rebuild_ctr[4], 1u);
+  }
 
-  // 5. the CTA that finishes last packs the var blocks into the image and writes the headers
+  // 5. the CTA that finishes last publishes the totals and resets the counters
   __threadfence();
   __syncthreads();
   if (tid == 0) {
-    uint32_t ticket = atomicAdd(c.done_ctr, 1u);
+    uint32_t ticket = atomicAdd(&c.rebuild_ctr[0], 1u);
     s_last = (ticket == gridDim.x - 1);
   }
   __syncthreads();
-  if (!s_last) return;
+  if (!s_last || tid != 0) return;
   __threadfence();
-
-  const uint32_t T = c.n_tasks;
-  uint4 *hdr = reinterpret_cast<uint4 *>(c.image);
-  uint2 *slow = reinterpret_cast<uint2 *>(c.image + image_slow_offset(T));
-  const uint32_t dummy = image_dummy_offset(T), var0 = image_var_offset(T);
-  // headers of a task without index: everything points at the dummy block, where the
-  // bitmap reads 0 and T2 reads 0xFF ("nothing found")
-  const uint4 dummy_hdr = make_uint4(dummy, dummy, dummy + 64u, 0u);
-  if (tid < 32) {                               // dummy block, the out-of-range entry and its SLO row
-    reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid < 16 ? 0u : 0xFFFFFFFFu;
-    if (tid == 0) {
-      uint4 h = dummy_hdr;
-      h.z |= HDR_FLAG_INVALID << 21;
-      hdr[T] = h;
-      slow[T] = make_uint2(0u, 0u);
-    }
-  }
-  {
-    uint32_t *row = reinterpret_cast<uint32_t *>(c.image + image_slo_offset(T)) + T * SLO_BUCKETS;
-    for (uint32_t j = tid; j < SLO_BUCKETS; j += B) row[j] = 0u;
-  }
-  // 5a. var offsets = exclusive prefix sum of the var-block sizes (chunks of B tasks)
-  uint32_t carry = 0, longest = 0, entries = 0, not_indexed = 0;
-  __shared__ uint32_t scan_buf[1024];
-  __shared__ uint32_t s_copy_end;
-  bool overflow = var0 > c.image_capacity;
-  for (uint32_t t0 = 0; t0 < T; t0 += B) {
-    const uint32_t tt = t0 + tid;
-    const uint32_t len = tt < T ? __ldcg(c.f_len + tt) : 0u;
-    const uint32_t vbytes = tt < T ? __ldcg(c.f_var_bytes + tt) : 0u;
-    scan_buf[tid] = vbytes;
-    __syncthreads();
-    for (uint32_t o = 1; o < B; o <<= 1) {      // Hillis-Steele inclusive scan
-      uint32_t v = tid >= o ? scan_buf[tid - o] : 0u;
-      __syncthreads();
-      scan_buf[tid] += v;
-      __syncthreads();
-    }
-    const uint32_t chunk_total = scan_buf[B - 1];
-    const uint32_t incl = scan_buf[tid];
-    __syncthreads();                                               // scan_buf is reused below
-    if (var0 + carry + chunk_total > c.image_capacity) overflow = true;   // uniform
-    const uint32_t off = var0 + carry + incl - vbytes;             // from the start of the image
-    // a block that does not end below what the 18-bit offsets can address is left out: the
-    // task is then served by the slow path, like one whose list is too long for the index
-    const bool addressable = off + vbytes <= IMAGE_OFFSET_LIMIT;
-    if (tt < T && !overflow) {
-      uint4 h = dummy_hdr;
-      uint2 sl = make_uint2(0u, len > 255u ? 0u : len);
-      if (len == 0) {
-        h.z |= HDR_FLAG_INVALID << 21;
-      } else if (vbytes == 0 || !addressable) {
-        h.z |= HDR_FLAG_NOT_INDEXED << 21;
-        ++not_indexed;
-      } else {
-        const uint4 rel = __ldcg(c.f_hdr + tt);
-        const uint2 srel = __ldcg(c.f_slow + tt);
-        h = make_uint4(rel.x + off, rel.y + off, rel.z + off, rel.w);
-        sl = make_uint2(srel.x + off, srel.y);
-      }
-      hdr[tt] = h;
-      slow[tt] = sl;
-    }
-    // offsets stay ascending: empty blocks share the next block's offset, and the blocks
-    // that are left out (and the padding past T) form a suffix of sentinels
-    scan_buf[tid] = (tt < T && addressable) ? off : 0xFFFFFFFFu;
-    if (tid == 0) s_copy_end = var0 + carry;
-    __syncthreads();
-    if (tt < T && addressable && vbytes) atomicMax(&s_copy_end, off + vbytes);
-    __syncthreads();
-    // 5b. copy this chunk's var blocks: 16-byte units spread over all threads; a unit finds
-    // its block by binary search over the chunk's ascending offsets
-    if (!overflow) {
-      const uint32_t first = var0 + carry;
-      const uint32_t units = (s_copy_end - first) >> 4;
-      const uint4 *reg4 = reinterpret_cast<const uint4 *>(c.regions);
-      uint4 *img4 = reinterpret_cast<uint4 *>(c.image);
-      for (uint32_t u0 = 0; u0 < units; u0 += 4u * B) {
-        uint4 v[4];
-        uint32_t dst[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t u = u0 + (uint32_t)j * B + tid;
-          dst[j] = 0xFFFFFFFFu;
-          if (u < units) {
-            const uint32_t byte = first + (u << 4);
-            uint32_t lo = 0, hi = B;                    // last i with scan_buf[i] <= byte
-            while (hi - lo > 1) {
-              const uint32_t mid = (lo + hi) >> 1;
-              if (scan_buf[mid] <= byte) lo = mid; else hi = mid;
-            }
-            const uint32_t tsrc = t0 + lo;
-            const uint32_t Vt = __ldg(c.task_off + tsrc + 1) - __ldg(c.task_off + tsrc);
-            const uint32_t src_byte = __ldg(c.reg_off + tsrc) + region_var_offset(Vt) + (byte - scan_buf[lo]);
-            v[j] = __ldcg(reg4 + (src_byte >> 4));
-            dst[j] = byte >> 4;
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          if (dst[j] != 0xFFFFFFFFu) img4[dst[j]] = v[j];
-      }
-    }
-    longest = max(longest, len);
-    entries += len;
-    __syncthreads();
-    carry += chunk_total;
-  }
-  // totals for reporting
-  longest = __reduce_max_sync(0xFFFFFFFFu, longest);
-  entries = __reduce_add_sync(0xFFFFFFFFu, entries);
-  not_indexed = __reduce_add_sync(0xFFFFFFFFu, not_indexed);
-  __shared__ uint32_t tot[3];
-  if (tid == 0) tot[0] = tot[1] = tot[2] = 0;
-  __syncthreads();
-  if ((tid & 31) == 0) { atomicMax(&tot[0], longest); atomicAdd(&tot[1], entries); atomicAdd(&tot[2], not_indexed); }
-  __syncthreads();
-  if (tid == 0) {
-    if (overflow) atomicMax(c.err, (uint32_t)DEV_ERR_IMAGE_OVERFLOW);
-    c.image_hdr[0] = overflow ? 0xFFFFFFFFu : var0 + carry;
-    c.image_hdr[1] = tot[0];
-    c.image_hdr[2] = tot[1];
-    c.image_hdr[3] = tot[2];
-    *c.done_ctr = 0;
-  }
+  volatile uint32_t *ctr = c.rebuild_ctr;
+  c.image_hdr[0] = image_var_offset(c.n_tasks) + ctr[1];
+  c.image_hdr[1] = ctr[2];
+  c.image_hdr[2] = ctr[3];
+  c.image_hdr[3] = ctr[4];
+  ctr[0] = 0; ctr[1] = 0; ctr[2] = 0; ctr[3] = 0; ctr[4] = 0;
 }
 
 }  // namespace
