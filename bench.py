@@ -39,7 +39,7 @@ NCU_TRAFFIC_BYTES_PER_QUERY = None
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3", choices=["C2", "C3", "C4", "C5"])
@@ -105,7 +105,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.004)
+            time.sleep(0.001)
 
     def __enter__(self):
         if self._h is not None:
@@ -156,7 +156,7 @@ def cpu_baseline(w, target_s: float = 12.0) -> dict:
     dt = time.perf_counter() - t0
     return {"value": n / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"first {n} of {w.n_queries} queries of {w.name}, select + load update, "
-                      f"{dt:.1f} s"}
+                      f"{dt:.1f} s wall on {threads} threads ({dt * threads:.0f} core-seconds)"}
 
 
 def run_reference(args):
