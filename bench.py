@@ -30,10 +30,11 @@ METRIC = "queries decided/sec"
 UNIT = "queries/s"
 ALGO_BYTES_PER_QUERY = 12          # 2 (task) + 4 (slo) + 2 (min acc) read, 4 (decision) written
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one selection-kernel launch, from the ncu
-# capture summarised under profiles/ (bytes per query x queries of a launch); None until a
-# capture of the current kernel exists.
-NCU_TRAFFIC_BYTES_PER_QUERY = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one selection-kernel launch on the 2^24-query
+# workload, from the ncu capture summarised in profiles/select_kernel_C3.md, per query (part of
+# the decisions is still in L2 when the kernel ends, hence below 12 B).  Set to None when the
+# kernel changes until the counters are taken again.
+NCU_TRAFFIC_BYTES_PER_QUERY = (134.47e6 + 20.56e6) / (1 << 24)
 
 
 def parse_args():
