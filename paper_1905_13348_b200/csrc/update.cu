@@ -87,14 +87,27 @@ tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_
   __syncthreads();
   uint32_t n_feas = 0, n_nofeas = 0, n_inval = 0;
   auto one = [&](uint32_t d) {
-    if (d < n_variants) { atomicAdd(&hist[d], 1u); ++n_feas; }   // d < n_variants < 2^31: bit 31 clear
-    else if (d != INFAAS_INVALID && (d & INFAAS_NO_FEASIBLE)) ++n_nofeas;
-    else ++n_inval;
+    const bool feas = d < n_variants;                            // d < n_variants < 2^31: bit 31 clear
+    const bool nofeas = !feas && d != INFAAS_INVALID && (d >> 31);
+    if (feas) atomicAdd(&hist[d], 1u);
+    n_feas += feas;
+    n_nofeas += nofeas;
+    n_inval += !feas && !nofeas;
   };
   const uint64_t n4 = n >> 2;
   const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
   const uint4 *dec4 = reinterpret_cast<const uint4 *>(decision);
-  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+  // four 128-bit loads in flight per thread: the loop is bound by load latency otherwise
+  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < n4; i += 4 * stride) {
+    const uint4 d0 = __ldcs(dec4 + i), d1 = __ldcs(dec4 + i + stride);
+    const uint4 d2 = __ldcs(dec4 + i + 2 * stride), d3 = __ldcs(dec4 + i + 3 * stride);
+    one(d0.x); one(d0.y); one(d0.z); one(d0.w);
+    one(d1.x); one(d1.y); one(d1.z); one(d1.w);
+    one(d2.x); one(d2.y); one(d2.z); one(d2.w);
+    one(d3.x); one(d3.y); one(d3.z); one(d3.w);
+  }
+  for (; i < n4; i += stride) {
     const uint4 d = __ldcs(dec4 + i);
     one(d.x); one(d.y); one(d.z); one(d.w);
   }
