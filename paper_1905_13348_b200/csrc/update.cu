@@ -168,7 +168,7 @@ constexpr uint32_t BITS_OF_2_POW_32 = 0x4F800000u;
 struct IndexScratch {          // shared memory used while building one task's index
   uint32_t pred[256], Pd[256], ids[256];
   uint16_t acc[256], Ad[256];
-  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256];
+  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256], bucket[256];
   uint32_t ks, ka, base;
 };
 
@@ -181,45 +181,82 @@ __device__ __forceinline__ void write_header(const DeviceCatalog &c, uint32_t t,
   if (threadIdx.x < HDR_BYTES / 16u) reinterpret_cast<uint4 *>(c.image + HDR_BYTES * t)[threadIdx.x] = h;
 }
 
+// Sum / OR over the aligned group of 8 lanes this lane belongs to.
+__device__ __forceinline__ uint32_t group8_add(uint32_t v) {
+  v += __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+  v += __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+  v += __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+  return v;
+}
+__device__ __forceinline__ uint32_t group8_or(uint32_t v) {
+  v |= __shfl_xor_sync(0xFFFFFFFFu, v, 1);
+  v |= __shfl_xor_sync(0xFFFFFFFFu, v, 2);
+  v |= __shfl_xor_sync(0xFFFFFFFFu, v, 4);
+  return v;
+}
+
 // Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh) into
 // a block of the image obtained from the block cursor.  S.pred / S.acc / S.ids hold the
 // list in scan order.  Returns false (all threads) if the list cannot be indexed: its
 // accuracies span more than the bitmap supports, or the block lies beyond what the 16-bit
-// offsets address.
+// offsets address.  blockDim = REBUILD_THREADS: the pair loops give every entry 8 lanes, and
+// the tables, which do not depend on each other, are written by different groups of warps.
 __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, IndexScratch &S) {
   const uint32_t tid = threadIdx.x, B = blockDim.x;
-  // distinct values and their ranks
-  for (uint32_t p = tid; p < F; p += B) {
-    bool fp = true, fa = true;
-    for (uint32_t q = 0; q < p; ++q) {
-      fp &= S.pred[q] != S.pred[p];
-      fa &= S.acc[q] != S.acc[p];
+  const uint32_t sub = tid & 7u, PB = B >> 3;          // lane of the entry's group; entries per pass
+  // distinct values ...
+  for (uint32_t p0 = 0; p0 < F; p0 += PB) {            // uniform trip count
+    const uint32_t p = p0 + (tid >> 3);
+    uint32_t dup = 0;                                  // bit 0: an earlier entry has this latency; bit 1: accuracy
+    if (p < F) {
+      const uint32_t pp = S.pred[p], pa = S.acc[p];
+      for (uint32_t q = sub; q < p; q += 8) dup |= (S.pred[q] == pp ? 1u : 0u) | (S.acc[q] == pa ? 2u : 0u);
     }
-    S.firstP[p] = fp;
-    S.firstA[p] = fa;
+    dup = group8_or(dup);
+    if (p < F && sub == 0) { S.firstP[p] = !(dup & 1u); S.firstA[p] = !(dup & 2u); }
   }
   if (tid == 0) { S.ks = 0; S.ka = 0; }
   __syncthreads();
-  for (uint32_t p = tid; p < F; p += B) {
-    uint32_t rp = 0, ra = 0;
-    for (uint32_t q = 0; q < F; ++q) {
-      rp += S.firstP[q] && S.pred[q] < S.pred[p];
-      ra += S.firstA[q] && S.acc[q] < S.acc[p];
+  // ... and their ranks
+  for (uint32_t p0 = 0; p0 < F; p0 += PB) {
+    const uint32_t p = p0 + (tid >> 3);
+    uint32_t cnt = 0;                                  // latency rank | accuracy rank << 16
+    if (p < F) {
+      const uint32_t pp = S.pred[p], pa = S.acc[p];
+      for (uint32_t q = sub; q < F; q += 8)
+        cnt += ((S.firstP[q] && S.pred[q] < pp) ? 1u : 0u) + ((S.firstA[q] && S.acc[q] < pa) ? 0x10000u : 0u);
     }
-    S.idxP[p] = (unsigned char)rp;
-    S.idxA[p] = (unsigned char)ra;
-    S.Pd[rp] = S.pred[p];
-    S.Ad[ra] = S.acc[p];
-    atomicMax(&S.ks, rp + 1);
-    atomicMax(&S.ka, ra + 1);
+    cnt = group8_add(cnt);
+    if (p < F && sub == 0) {
+      const uint32_t rp = cnt & 0xFFFFu, ra = cnt >> 16;
+      S.idxP[p] = (unsigned char)rp;
+      S.idxA[p] = (unsigned char)ra;
+      S.Pd[rp] = S.pred[p];
+      S.Ad[ra] = S.acc[p];
+      atomicMax(&S.ks, rp + 1);
+      atomicMax(&S.ka, ra + 1);
+    }
   }
   __syncthreads();
   const uint32_t Ks = S.ks, Ka = S.ka;
+  // SLO buckets: they cover the list's latencies up to SLO_CAP_US; larger ones share bucket 255
+  const uint32_t clo = float_bits(S.Pd[0]) >> 16;
+  const uint32_t chi = max(clo, float_bits(min(S.Pd[Ks - 1], SLO_CAP_US)) >> 16);
+  uint32_t sh = 0;
+  while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
+  const uint32_t bmin = clo >> sh, Sh = 16u + sh;
+  for (uint32_t i = tid; i < Ks; i += B)
+    S.bucket[i] = (unsigned char)(min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1));
   // positions ordered by rank of pred_lat (ties in scan order)
-  for (uint32_t p = tid; p < F; p += B) {
+  for (uint32_t p0 = 0; p0 < F; p0 += PB) {
+    const uint32_t p = p0 + (tid >> 3);
     uint32_t o = 0;
-    for (uint32_t q = 0; q < F; ++q) o += S.idxP[q] < S.idxP[p] || (S.idxP[q] == S.idxP[p] && q < p);
-    S.order[o] = (unsigned char)p;
+    if (p < F) {
+      const uint32_t ip = S.idxP[p];
+      for (uint32_t q = sub; q < F; q += 8) o += S.idxP[q] < ip || (S.idxP[q] == ip && q < p);
+    }
+    o = group8_add(o);
+    if (p < F && sub == 0) S.order[o] = (unsigned char)p;
   }
 
   // block layout and its place in the image
@@ -240,81 +277,32 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   const uint32_t base = S.base;
   if (base == 0xFFFFFFFFu) return false;
   unsigned char *blk = c.image + base;
-
-  // ids, reversed; the slot of "position F" holds PENDING
-  uint32_t *ids_end = reinterpret_cast<uint32_t *>(blk + BL.t2);
-  for (uint32_t p = tid; p <= F; p += B) ids_end[-1 - (int)p] = p < F ? S.ids[p] : PENDING;
-
-  // T2, one thread per accuracy rank k: walk the positions in latency-rank order
-  unsigned char *T2 = blk + BL.t2;
-  for (uint32_t k = tid; k < width; k += B) {
-    uint32_t cur = F, o = 0;
-    T2[k] = (unsigned char)F;                                  // r = 0: no latency is met
-    for (uint32_t r = 1; r <= Ks; ++r) {
-      while (o < F && S.idxP[S.order[o]] == r - 1) {
-        const uint32_t p = S.order[o];
-        if (S.idxA[p] >= k && p < cur) cur = p;
-        ++o;
-      }
-      T2[r * width + k] = (unsigned char)cur;
-    }
-    T2[(Ks + 1u) * width + k] = (unsigned char)F;
-  }
-
-  // accuracy bitmap with running popcounts
-  uint32_t *bitmap = reinterpret_cast<uint32_t *>(blk + BL.bitmap);
-  for (uint32_t w = tid; w < nbw; w += B) {
-    uint32_t bits = 0, prefix = 0;
-    for (uint32_t i = 0; i < Ka; ++i) {
-      const uint32_t x = S.Ad[i] - acc_lo, xw = x / ACC_WORD_BITS;
-      prefix += xw < w;
-      if (xw == w) bits |= 1u << (x - xw * ACC_WORD_BITS);
-    }
-    bitmap[w] = (prefix << 24) | bits;
-  }
-
-  // what the nearest-miss search reads
   unsigned char *slow = blk + BL.slow;
-  uint2 *walk = reinterpret_cast<uint2 *>(slow + SL.walk);
-  for (uint32_t o = tid; o < F; o += B) {
-    const uint32_t p = S.order[o];
-    walk[o] = make_uint2(S.pred[p], (uint32_t)S.acc[p] | (p << 16));
-  }
-  uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
-  for (uint32_t i = tid; i < Ks; i += B) Pd_g[i] = S.Pd[i];
-  uint32_t *bestA = reinterpret_cast<uint32_t *>(slow + SL.bestA);
-  for (uint32_t r = tid; r <= Ks; r += B) {
-    uint32_t best = 0xFFu, best_acc = 0, cnt = 0;               // highest accuracy among ranks < r
-    for (uint32_t p = 0; p < F; ++p) {
-      if (S.idxP[p] < r) {
-        ++cnt;
-        if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
-      }
-    }
-    bestA[r] = best_acc | (best << 16);
-    slow[SL.ordStart + r] = (unsigned char)cnt;
-  }
-  uint2 *bestB = reinterpret_cast<uint2 *>(slow + SL.bestB);
-  for (uint32_t k = tid; k <= Ka; k += B) {
-    uint32_t best = 0xFFu, best_pred = 0;                        // lowest latency among accuracy ranks >= k
-    for (uint32_t p = 0; p < F; ++p) {
-      if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
-    }
-    bestB[k] = make_uint2(best_pred, best);
-  }
 
-  // SLO records.  The buckets cover the list's latencies up to SLO_CAP_US; larger ones
-  // share bucket 255.
-  const uint32_t clo = float_bits(S.Pd[0]) >> 16;
-  const uint32_t chi = max(clo, float_bits(min(S.Pd[Ks - 1], SLO_CAP_US)) >> 16);
-  uint32_t sh = 0;
-  while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
-  const uint32_t bmin = clo >> sh, Sh = 16u + sh;
+  // From here on nothing depends on anything else: thread ranges take one table each.
+  // [lo, lo + n) of the CTA's threads run `body(x)` for x = 0 .. count - 1.
+  auto share = [&](uint32_t lo, uint32_t n, uint32_t count, auto body) {
+    if (tid >= lo && tid < lo + n)
+      for (uint32_t x = tid - lo; x < count; x += n) body(x);
+  };
+
+  // T2: cell (r, k) = first position whose latency rank is < r and accuracy rank >= k
+  unsigned char *T2 = blk + BL.t2;
+  share(0, B / 2, (Ks + 2u) * width, [&](uint32_t cell) {
+    const uint32_t r = cell / width, k = cell - r * width;
+    uint32_t pos = F;
+    if (r >= 1 && r <= Ks)
+      for (uint32_t p = 0; p < F; ++p)
+        if (S.idxP[p] < r && S.idxA[p] >= k) { pos = p; break; }
+    T2[cell] = (unsigned char)pos;
+  });
+
+  // SLO records (see common.cuh)
   uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
-  for (uint32_t j = tid; j < SLO_BUCKETS; j += B) {
+  share(B / 2, B / 4, SLO_BUCKETS, [&](uint32_t j) {
     uint32_t lb = 0, cnt = 0, thr = 0;
     for (uint32_t i = 0; i < Ks; ++i) {
-      const uint32_t b = min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1);
+      const uint32_t b = S.bucket[i];
       lb += b < j;
       if (b == j) { ++cnt; thr = S.Pd[i]; }
     }
@@ -328,7 +316,51 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
       r = thr <= lo ? (lb + 1u) << 24 : (lb << 24) | (0x00FFFFFFu - ((thr - 1u) & 0x00FFFFFFu));
     }
     rec[j] = r;
-  }
+  });
+
+  // accuracy bitmap with running popcounts
+  uint32_t *bitmap = reinterpret_cast<uint32_t *>(blk + BL.bitmap);
+  share(3 * B / 4, B / 8, nbw, [&](uint32_t w) {
+    uint32_t bits = 0, prefix = 0;
+    for (uint32_t i = 0; i < Ka; ++i) {
+      const uint32_t x = S.Ad[i] - acc_lo, xw = x / ACC_WORD_BITS;
+      prefix += xw < w;
+      if (xw == w) bits |= 1u << (x - xw * ACC_WORD_BITS);
+    }
+    bitmap[w] = (prefix << 24) | bits;
+  });
+
+  // what the nearest-miss search reads
+  uint32_t *bestA = reinterpret_cast<uint32_t *>(slow + SL.bestA);
+  share(7 * B / 8, B / 16, Ks + 1u, [&](uint32_t r) {
+    uint32_t best = 0xFFu, best_acc = 0, cnt = 0;               // highest accuracy among ranks < r
+    for (uint32_t p = 0; p < F; ++p) {
+      if (S.idxP[p] < r) {
+        ++cnt;
+        if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
+      }
+    }
+    bestA[r] = best_acc | (best << 16);
+    slow[SL.ordStart + r] = (unsigned char)cnt;
+  });
+  uint2 *bestB = reinterpret_cast<uint2 *>(slow + SL.bestB);
+  share(15 * B / 16, B / 16, Ka + 1u, [&](uint32_t k) {
+    uint32_t best = 0xFFu, best_pred = 0;                        // lowest latency among accuracy ranks >= k
+    for (uint32_t p = 0; p < F; ++p) {
+      if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
+    }
+    bestB[k] = make_uint2(best_pred, best);
+  });
+  // small copies, after the short loops above
+  uint32_t *ids_end = reinterpret_cast<uint32_t *>(blk + BL.t2);   // ids, reversed; slot F holds PENDING
+  share(3 * B / 4, B / 8, F + 1u, [&](uint32_t p) { ids_end[-1 - (int)p] = p < F ? S.ids[p] : PENDING; });
+  uint2 *walk = reinterpret_cast<uint2 *>(slow + SL.walk);
+  share(7 * B / 8, B / 16, F, [&](uint32_t o) {
+    const uint32_t p = S.order[o];
+    walk[o] = make_uint2(S.pred[p], (uint32_t)S.acc[p] | (p << 16));
+  });
+  uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
+  share(15 * B / 16, B / 16, Ks, [&](uint32_t i) { Pd_g[i] = S.Pd[i]; });
 
   const uint32_t cb = ((base + BL.bitmap) >> 2) - acc_lo / ACC_WORD_BITS;
   write_header(c, t, make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
@@ -337,7 +369,11 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   return true;
 }
 
-__global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us) {
+constexpr uint32_t REBUILD_THREADS = 1024;
+constexpr uint32_t RANK_SORT_MAX = 512;   // tasks up to this size are sorted by counting smaller keys
+
+__global__ void __launch_bounds__(REBUILD_THREADS)
+rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long *k64 = reinterpret_cast<unsigned long long *>(smem_raw);   // cost<<32 | pred
   uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
@@ -385,43 +421,75 @@ __global__ void rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, ui
   }
   __syncthreads();
 
-  // 2. bitonic sort of P keys, ascending in (cost, pred, 10000-acc, local index)
-  for (uint32_t k = 2; k <= P; k <<= 1) {
-    for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-      for (uint32_t x = tid; x < (P >> 1); x += B) {
-        uint32_t i = ((x & ~(j - 1)) << 1) | (x & (j - 1));   // lower index of the pair
-        uint32_t l = i | j;
-        bool up = (i & k) == 0;
-        unsigned long long a64 = k64[i], b64 = k64[l];
-        uint32_t a32 = k32[i], b32 = k32[l];
-        bool swap = up ? key_less(b64, b32, a64, a32) : key_less(a64, a32, b64, b32);
-        if (swap) {
-          k64[i] = b64; k64[l] = a64;
-          k32[i] = b32; k32[l] = a32;
-        }
-      }
-      __syncthreads();
-    }
-  }
-
-  // 3. prune.  In sorted order every dominator of p sits before p, and every earlier entry
-  // q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not larger by the
-  // sort, and it differs in some attribute or has the smaller id).
   uint32_t my_kept = 0;
-  for (uint32_t p = tid; p < V; p += B) {
-    const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
-    bool kp = true;
-    for (uint32_t q0 = 0; q0 < p && kp; q0 += 8) {     // groups of 8, exit between groups
-      bool dom = false;
-#pragma unroll
-      for (uint32_t j = 0; j < 8; ++j) {
-        const uint32_t q = min(q0 + j, p - 1);          // clamped repeats are harmless
-        dom |= (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
+  if (sort_n <= RANK_SORT_MAX) {
+    // 2+3 (small tasks).  Rank sort fused with the prune: entry q sorts before p iff its key
+    // (cost, pred, 10000-acc, local index) is smaller, and it dominates p iff in addition
+    // pred_q <= pred_p and acc_q >= acc_p (its cost is not larger by the key order, and it
+    // differs in some attribute or has the smaller id).  G lanes share an entry's comparisons.
+    unsigned long long *o64 = reinterpret_cast<unsigned long long *>(keep + sort_n + ((8u - ((13u * sort_n) & 7u)) & 7u));
+    uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);
+    const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
+    uint32_t rank = 0, dom = 0;
+    unsigned long long a64 = 0;
+    uint32_t a32 = 0;
+    if (p < V) {
+      a64 = k64[p]; a32 = k32[p];
+      const uint32_t pred_p = (uint32_t)a64, inv_p = a32 >> 16;
+      for (uint32_t q = sidx; q < V; q += G) {
+        const unsigned long long b64 = k64[q];
+        const uint32_t b32 = k32[q];
+        const bool less = key_less(b64, b32, a64, a32);
+        rank += less;
+        dom |= (less && (uint32_t)b64 <= pred_p && (b32 >> 16) <= inv_p) ? 1u : 0u;
       }
-      kp = !dom;
     }
-    keep[p] = kp;
-    my_kept += kp;
+    for (uint32_t o = G >> 1; o; o >>= 1) {            // G is a power of two, groups are lane-aligned
+      rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+      dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);
+    }
+    if (p < V && sidx == 0) {
+      o64[rank] = a64; o32[rank] = a32; keep[rank] = !dom;
+      my_kept = !dom;
+    }
+    k64 = o64; k32 = o32;
+  } else {
+    // 2. bitonic sort of P keys, ascending in (cost, pred, 10000-acc, local index)
+    for (uint32_t k = 2; k <= P; k <<= 1) {
+      for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+        for (uint32_t x = tid; x < (P >> 1); x += B) {
+          uint32_t i = ((x & ~(j - 1)) << 1) | (x & (j - 1));   // lower index of the pair
+          uint32_t l = i | j;
+          bool up = (i & k) == 0;
+          unsigned long long a64 = k64[i], b64 = k64[l];
+          uint32_t a32 = k32[i], b32 = k32[l];
+          bool swap = up ? key_less(b64, b32, a64, a32) : key_less(a64, a32, b64, b32);
+          if (swap) {
+            k64[i] = b64; k64[l] = a64;
+            k32[i] = b32; k32[l] = a32;
+          }
+        }
+        __syncthreads();
+      }
+    }
+    // 3. prune.  In sorted order every dominator of p sits before p, and every earlier entry
+    // q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not larger by the
+    // sort, and it differs in some attribute or has the smaller id).
+    for (uint32_t p = tid; p < V; p += B) {
+      const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
+      bool kp = true;
+      for (uint32_t q0 = 0; q0 < p && kp; q0 += 8) {     // groups of 8, exit between groups
+        bool dom = false;
+#pragma unroll
+        for (uint32_t j = 0; j < 8; ++j) {
+          const uint32_t q = min(q0 + j, p - 1);          // clamped repeats are harmless
+          dom |= (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
+        }
+        kp = !dom;
+      }
+      keep[p] = kp;
+      my_kept += kp;
+    }
   }
   if (tid == 0) s_total = 0;
   __syncthreads();
@@ -529,9 +597,9 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream) {
   uint32_t P = 1;
   while (P < c.max_task_variants) P <<= 1;
-  uint32_t block = P < 256 ? 256 : (P > 1024 ? 1024 : P);
-  size_t smem = (size_t)P * 13;
-  rebuild_kernel<<<c.n_tasks, block, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
+  // small tasks: room for the rank sort's second copy of the keys (12 bytes per entry, 8-byte aligned)
+  size_t smem = (size_t)P * 13 + (P <= RANK_SORT_MAX ? (size_t)P * 12 + 8 : 0);
+  rebuild_kernel<<<c.n_tasks, REBUILD_THREADS, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
   return cudaGetLastError();
 }
 
