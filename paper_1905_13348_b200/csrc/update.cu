@@ -85,33 +85,35 @@ tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_
   for (uint32_t i = threadIdx.x; i < n_variants; i += blockDim.x) hist[i] = 0;
   if (threadIdx.x < 3) blk[threadIdx.x] = 0;
   __syncthreads();
-  uint32_t n_feas = 0, n_nofeas = 0, n_inval = 0;
+  // per decision: one compare + predicated shared-memory atomic, and two counters; invalid
+  // decisions are what remains of the total
+  uint32_t n_feas = 0, n_nofeas = 0, n_seen = 0;
   auto one = [&](uint32_t d) {
-    const bool feas = d < n_variants;                            // d < n_variants < 2^31: bit 31 clear
-    const bool nofeas = !feas && d != INFAAS_INVALID && (d >> 31);
-    if (feas) atomicAdd(&hist[d], 1u);
-    n_feas += feas;
-    n_nofeas += nofeas;
-    n_inval += !feas && !nofeas;
+    if (d < n_variants) atomicAdd(&hist[d], 1u);                 // d < n_variants < 2^31: bit 31 clear
+    n_feas += d < n_variants;
+    n_nofeas += (d - INFAAS_NO_FEASIBLE) < 0x7FFFFFFFu;          // bit 31 set and not INFAAS_INVALID
   };
-  const uint64_t n4 = n >> 2;
-  const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+  const uint32_t n4 = (uint32_t)(n >> 2);                        // n <= 2^32 - 1 (checked by the caller)
+  const uint32_t stride = gridDim.x * blockDim.x;
   const uint4 *dec4 = reinterpret_cast<const uint4 *>(decision);
-  // four 128-bit loads in flight per thread: the loop is bound by load latency otherwise
-  uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  for (; i + 3 * stride < n4; i += 4 * stride) {
+  // four 128-bit loads in flight per thread
+  uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  for (; n4 >= 3 * stride && i < n4 - 3 * stride; i += 4 * stride) {
     const uint4 d0 = __ldcs(dec4 + i), d1 = __ldcs(dec4 + i + stride);
     const uint4 d2 = __ldcs(dec4 + i + 2 * stride), d3 = __ldcs(dec4 + i + 3 * stride);
     one(d0.x); one(d0.y); one(d0.z); one(d0.w);
     one(d1.x); one(d1.y); one(d1.z); one(d1.w);
     one(d2.x); one(d2.y); one(d2.z); one(d2.w);
     one(d3.x); one(d3.y); one(d3.z); one(d3.w);
+    n_seen += 16;
   }
   for (; i < n4; i += stride) {
     const uint4 d = __ldcs(dec4 + i);
     one(d.x); one(d.y); one(d.z); one(d.w);
+    n_seen += 4;
   }
-  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) one(decision[(n4 << 2) + threadIdx.x]);
+  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) { one(decision[((uint64_t)n4 << 2) + threadIdx.x]); ++n_seen; }
+  uint32_t n_inval = n_seen - n_feas - n_nofeas;
   n_feas = __reduce_add_sync(0xFFFFFFFFu, n_feas);
   n_nofeas = __reduce_add_sync(0xFFFFFFFFu, n_nofeas);
   n_inval = __reduce_add_sync(0xFFFFFFFFu, n_inval);
