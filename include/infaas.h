@@ -118,6 +118,26 @@ int infaas_select_batch(infaas_catalog *c, const uint16_t *d_task, const uint32_
 int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n,
                        uint32_t window_us, void *cuda_stream);
 
+/* The two halves of infaas_load_update, for windows whose queries are shared out over several
+ * GPUs (Section 4.2.2 and Section 5: every worker's monitoring daemon reports the load it saw;
+ * the load of a variant is the sum over the workers).  Each GPU holds the same catalog and
+ * decides its share of the window; then
+ *     infaas_tally           adds the share's decisions to the pending per-variant counts,
+ *     infaas_pending_counts  copies the pending counts out (set = 0) -- sum them over the
+ *                            GPUs, e.g. with an all-reduce -- and back in (set = 1),
+ *     infaas_advance         applies the queue recursion with the pending counts, clears
+ *                            them and rebuilds the scan lists, as infaas_load_update does.
+ * infaas_load_update(c, d, n, w, s) equals infaas_tally(c, d, n, s); infaas_advance(c, w, s).
+ * With the same summed counts every GPU reaches the same load state.  The counters of
+ * infaas_catalog_get_state stay local to each GPU (they count the decisions it tallied).
+ *   d_decision   as for infaas_load_update.
+ *   d_counts     DEVICE array of n_variants u32 indexed by variant id, 16-byte aligned;
+ *                written (set = 0) or read (set = 1).
+ * Asynchronous, stream-ordered, allocate nothing.  Errors: E_NULL, E_ALIGN, E_TOO_LARGE, E_CUDA. */
+int infaas_tally(infaas_catalog *c, const uint32_t *d_decision, uint64_t n, void *cuda_stream);
+int infaas_pending_counts(infaas_catalog *c, uint32_t *d_counts, int set, void *cuda_stream);
+int infaas_advance(infaas_catalog *c, uint32_t window_us, void *cuda_stream);
+
 /* Copy the load state to HOST arrays (any of the four may be NULL to skip it):
  *   h_queued[n_variants], h_pred_lat_us[n_variants], h_served_total[n_variants] indexed by
  *   variant id; h_counters[3] = feasible decisions tallied, NO_FEASIBLE decisions seen,

@@ -6,7 +6,8 @@ are resolved lazily and raise if the library has not been built.
 from . import workloads  # noqa: F401
 
 _BINDING = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
-            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_tally_static", "infaas_catalog_get_info", "Catalog", "InfaasError",
+            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_tally_static", "infaas_catalog_get_info",
+            "infaas_tally", "infaas_pending_counts", "infaas_advance", "Catalog", "InfaasError",
             "NO_FEASIBLE", "INVALID")
 
 

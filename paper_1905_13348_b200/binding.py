@@ -21,7 +21,8 @@ _lib = None
 
 EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
-           "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info")
+           "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info",
+           "infaas_tally", "infaas_pending_counts", "infaas_advance")
 
 
 class InfaasError(RuntimeError):
@@ -53,6 +54,11 @@ def _load():
     lib.infaas_catalog_free.restype = None
     for name in ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
                  "infaas_catalog_get_state", "infaas_catalog_get_frontier"):
+        getattr(lib, name).restype = i32
+    lib.infaas_tally.argtypes = [vp, vp, u64, vp]
+    lib.infaas_pending_counts.argtypes = [vp, vp, i32, vp]
+    lib.infaas_advance.argtypes = [vp, u32, vp]
+    for name in ("infaas_tally", "infaas_pending_counts", "infaas_advance"):
         getattr(lib, name).restype = i32
     lib.infaas_tally_static.argtypes = [vp, u64, u32, vp, vp, i32, vp]
     lib.infaas_tally_static.restype = i32
@@ -129,6 +135,24 @@ def infaas_load_update(cat: Catalog, d_decision, window_us: int, n=None, stream=
     n = int(d_decision.shape[0]) if n is None else int(n)
     _check(_load().infaas_load_update(cat.handle, _dev_ptr(d_decision, "u32"), n, int(window_us),
                                       _stream_ptr(stream)), "infaas_load_update")
+
+
+def infaas_tally(cat: Catalog, d_decision, n=None, stream=None) -> None:
+    n = int(d_decision.shape[0]) if n is None else int(n)
+    _check(_load().infaas_tally(cat.handle, _dev_ptr(d_decision, "u32"), n, _stream_ptr(stream)),
+           "infaas_tally")
+
+
+def infaas_pending_counts(cat: Catalog, d_counts, set: bool, stream=None) -> None:
+    """d_counts: int32/uint32 CUDA tensor of n_variants; written (set=False) or read (set=True)."""
+    if d_counts.numel() < cat.n_variants:
+        raise ValueError("d_counts is shorter than n_variants")
+    _check(_load().infaas_pending_counts(cat.handle, _dev_ptr(d_counts, "u32"), 1 if set else 0,
+                                         _stream_ptr(stream)), "infaas_pending_counts")
+
+
+def infaas_advance(cat: Catalog, window_us: int, stream=None) -> None:
+    _check(_load().infaas_advance(cat.handle, int(window_us), _stream_ptr(stream)), "infaas_advance")
 
 
 def infaas_catalog_get_state(cat: Catalog, stream=None) -> dict:

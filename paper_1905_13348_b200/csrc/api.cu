@@ -235,18 +235,41 @@ int infaas_select_batch(infaas_catalog *c, const uint16_t *d_task, const uint32_
   return INFAAS_OK;
 }
 
-int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n,
-                       uint32_t window_us, void *cuda_stream) {
+int infaas_tally(infaas_catalog *c, const uint32_t *d_decision, uint64_t n, void *cuda_stream) {
   if (!c) return INFAAS_E_NULL;
   if (n > 0xFFFFFFFFull) return INFAAS_E_TOO_LARGE;
   if (n > 0 && !d_decision) return INFAAS_E_NULL;
   if (n > 0 && !aligned16(d_decision)) return INFAAS_E_ALIGN;
   DeviceScope scope(c->device);
   if (scope.status != cudaSuccess) return cuda_fail(scope.status);
-  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  CUDA_TRY(infaas::launch_tally(c->d, d_decision, n, s));
-  CUDA_TRY(infaas::launch_rebuild(c->d, /*advance_queues=*/true, window_us, s));
+  CUDA_TRY(infaas::launch_tally(c->d, d_decision, n, static_cast<cudaStream_t>(cuda_stream)));
   return INFAAS_OK;
+}
+
+int infaas_pending_counts(infaas_catalog *c, uint32_t *d_counts, int set, void *cuda_stream) {
+  if (!c || !d_counts) return INFAAS_E_NULL;
+  if (!aligned16(d_counts)) return INFAAS_E_ALIGN;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  const size_t bytes = (size_t)c->d.n_variants * 4;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (set) CUDA_TRY(cudaMemcpyAsync(c->d.count_by_id, d_counts, bytes, cudaMemcpyDeviceToDevice, s));
+  else CUDA_TRY(cudaMemcpyAsync(d_counts, c->d.count_by_id, bytes, cudaMemcpyDeviceToDevice, s));
+  return INFAAS_OK;
+}
+
+int infaas_advance(infaas_catalog *c, uint32_t window_us, void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  CUDA_TRY(infaas::launch_rebuild(c->d, /*advance_queues=*/true, window_us, static_cast<cudaStream_t>(cuda_stream)));
+  return INFAAS_OK;
+}
+
+int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n,
+                       uint32_t window_us, void *cuda_stream) {
+  const int rc = infaas_tally(c, d_decision, n, cuda_stream);
+  return rc != INFAAS_OK ? rc : infaas_advance(c, window_us, cuda_stream);
 }
 
 int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_pred_lat_us,

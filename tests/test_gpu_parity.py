@@ -284,3 +284,44 @@ def test_full_size_windowed(name, state_every):
         assert int(o.counters.sum()) == w.n_queries
     finally:
         cat.free()
+
+
+def test_split_update_with_summed_counts_matches_whole_window():
+    """infaas_tally / infaas_pending_counts / infaas_advance: two catalogs on this GPU stand
+    in for two ranks; each decides its share of a window, the pending counts are summed and
+    handed to both, and both must reach the oracle's state for the whole window."""
+    import paper_1905_13348_b200 as P
+    from paper_1905_13348_b200 import sharding as S
+    torch = _torch()
+    w = W.make("C3", n_queries=5 * 8192, window=8192)
+    w.window_us = 300
+    cats = [P.infaas_catalog_load(w.rows, w.n_tasks) for _ in range(2)]
+    o = OracleCatalog(w.rows, w.n_tasks)
+    try:
+        for k in range(w.n_queries // w.window):
+            base = k * w.window
+            ws = slice(base, base + w.window)
+            want = o.select(w.task[ws], w.slo_us[ws], w.min_acc_bp[ws], 4)
+            o.load_update(want, w.window_us)
+            exported = []
+            for r, cat in enumerate(cats):
+                lo, hi = S.shard_bounds(w.window, 2, r)
+                sl = slice(base + lo, base + hi)
+                d_dec = gpu_select(cat, w.task[sl], w.slo_us[sl], w.min_acc_bp[sl])
+                assert np.array_equal(_to_host_u32(d_dec), want[lo:hi])
+                P.infaas_tally(cat, d_dec)
+                cnt = torch.zeros(w.n_variants, dtype=torch.int32, device="cuda")
+                P.infaas_pending_counts(cat, cnt, set=False)
+                exported.append(cnt)
+            total = exported[0] + exported[1]
+            for cat in cats:
+                P.infaas_pending_counts(cat, total, set=True)
+                P.infaas_advance(cat, w.window_us)
+                st = P.infaas_catalog_get_state(cat)
+                assert np.array_equal(st["queued"], o.queued)
+                assert np.array_equal(st["served_total"], o.served_total)
+                assert np.array_equal(st["pred_lat_us"], _np_pred(w.rows, o.queued))
+        assert o.queued.max() > 0
+    finally:
+        for cat in cats:
+            cat.free()
