@@ -157,7 +157,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_regions = carve((size_t)region_bytes);
   const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve((size_t)n_tasks * 16);
   const size_t o_image = carve((size_t)worst_image), o_hdr = carve(16);
-  const size_t o_counters = carve(24), o_rebuild = carve(32), o_err = carve(4);
+  const size_t o_counters = carve(24), o_rebuild = carve(32), o_err = carve(4), o_seen = carve(4);
 
 #define LOAD_TRY(expr)                                                     \
   do {                                                                     \
@@ -204,6 +204,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.counters = reinterpret_cast<unsigned long long *>(base + o_counters);
   d.rebuild_ctr = reinterpret_cast<uint32_t *>(base + o_rebuild);
   d.err = reinterpret_cast<uint32_t *>(base + o_err);
+  d.slo_seen = reinterpret_cast<uint32_t *>(base + o_seen);
   c->slot_of_id.swap(slot_of_id);
   c->task_off.swap(task_off);
   c->reg_off.swap(reg_off);

@@ -30,6 +30,8 @@ namespace infaas {
 //     exactly when slo >= thr;
 //   - otherwise R = Ks + 1, C = 0: row Ks + 1 of T2 holds only F, which sends the query to
 //     the exact slow path.
+// The buckets cover the list's latencies up to the largest SLO any batch has asked for so
+// far (kept as a bit mask, at least SLO_CAP_FLOOR_US); larger latencies share bucket 255.
 // k comes from a bitmap over accuracy values with running popcounts (24 bitmap bits and an
 // 8-bit prefix count per word), exact at one basis point.
 //
@@ -64,7 +66,7 @@ constexpr uint32_t ACC_WORD_BITS = 24;
 constexpr uint32_t MAX_ACC_WORDS = 255;          // nbw is an 8-bit field: 6120 basis points
 constexpr uint32_t HDR_BYTES = 128;              // 8 copies x 16 bytes
 constexpr uint32_t IMAGE_WORD_LIMIT = 1u << 16;  // t2_off / 4 and cb are 16-bit fields
-constexpr uint32_t SLO_CAP_US = 1u << 26;        // latencies above this share the last bucket
+constexpr uint32_t SLO_CAP_FLOOR_US = (1u << 20) - 1u;  // the buckets cover latencies at least up to here
 constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-2)
 
 constexpr uint32_t TASK_FLAG_INVALID = 1u;       // no variant: answer INFAAS_INVALID
@@ -155,6 +157,7 @@ struct DeviceCatalog {
   unsigned long long *counters;  // [3] feasible, no-feasible, invalid
   uint32_t *rebuild_ctr;         // [4] CTA arrival counter, block cursor, longest, entries (rebuild kernel)
   uint32_t *err;                 // sticky device error word (0 = fine)
+  uint32_t *slo_seen;            // OR of all SLOs the selection kernel has read
 };
 
 // Device error codes stored in DeviceCatalog::err.

@@ -293,9 +293,11 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
 
   // full tiles: 4 consecutive queries per lane, 128-bit loads, next tile prefetched (the
   // first tile was loaded by the caller while the image was being staged)
+  uint32_t slo_or = 0;                  // how large the SLOs get: sizes the buckets of later rebuilds
   for (uint32_t tile = warp; tile < full_tiles; tile += SELECT_WARPS) {
     const uint2 t = t4, a = a4;
     const uint4 s = s4;
+    slo_or |= s.x | s.y | s.z | s.w;
     const uint32_t next = tile + SELECT_WARPS;
     if (next < full_tiles) {
       const uint64_t i4 = (q0 + (uint64_t)next * WARP_TILE) / 4 + lane;
@@ -333,6 +335,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
         const uint64_t i = q0 + rel;
         const uint32_t tk = q.task[i], ac = q.min_acc[i];
         sq[0] = q.slo[i];
+        slo_or |= sq[0];
         ta[0] = tk | (ac << 16);
         d = decide_fast(img, n_tasks, rec_off, hdr_lane, tk, sq[0], ac);
         out[rel] = d;
@@ -343,6 +346,8 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
   }
   __syncwarp();
   resolve_parked(img, c, out, pk, 0, pk.cnt);
+  slo_or = __reduce_or_sync(0xFFFFFFFFu, slo_or);
+  if (lane == 0 && (slo_or & ~*c.slo_seen)) atomicOr(c.slo_seen, slo_or);
 }
 
 __global__ void __launch_bounds__(SELECT_THREADS, 1)

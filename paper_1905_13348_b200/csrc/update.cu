@@ -241,9 +241,12 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   }
   __syncthreads();
   const uint32_t Ks = S.ks, Ka = S.ka;
-  // SLO buckets: they cover the list's latencies up to SLO_CAP_US; larger ones share bucket 255
+  // SLO buckets: they cover the list's latencies up to the largest SLO asked for so far (as a
+  // bit mask: every SLO seen is <= cap); larger latencies share bucket 255
+  uint32_t cap = *c.slo_seen | SLO_CAP_FLOOR_US;
+  cap |= cap >> 1; cap |= cap >> 2; cap |= cap >> 4; cap |= cap >> 8; cap |= cap >> 16;
   const uint32_t clo = float_bits(S.Pd[0]) >> 16;
-  const uint32_t chi = max(clo, float_bits(min(S.Pd[Ks - 1], SLO_CAP_US)) >> 16);
+  const uint32_t chi = max(clo, float_bits(min(S.Pd[Ks - 1], cap)) >> 16);
   uint32_t sh = 0;
   while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
   const uint32_t bmin = clo >> sh, Sh = 16u + sh;
