@@ -82,8 +82,9 @@ inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) { return 
 
 // Byte offsets of the slow-path tables inside a task's block, relative to their start
 // (8-byte aligned), for a list of F entries with Ks / Ka distinct latencies / accuracies.
-//   walk[o]   uint2 (pred_lat, acc | position << 16), entries in ascending latency (ties
-//             in position order)
+//   walk[o]   uint2 (pred_lat, acc | position << 16): the "stair" entries -- those no other
+//             entry beats in both latency and accuracy -- in ascending latency (Fs <= F of
+//             them, all with different latencies; space for F)
 //   bestB[k]  uint2 (pred_lat, position) of the lowest-latency entry among those whose
 //             accuracy rank is >= k (first position among equals); position 0xFF if none
 //   Pd[i]     u32 distinct latencies
@@ -124,7 +125,7 @@ inline __host__ __device__ uint32_t block_capacity(uint32_t V) {
 inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_up_u32(12u * V, 64u); }
 
 // Slow-path parameters of a task (one uint4 per task, global memory).
-//   x = image offset of the slow tables   y = F | Ks << 8 | Ka << 16   z = flags   w = 0
+//   x = image offset of the slow tables   y = F | Ks << 8 | Ka << 16   z = flags   w = Fs
 // ---------------------------------------------------------------------------------------
 // Device catalog.  "Slot" order: variants bucketed by task, ascending id inside a task;
 // task t owns slots task_off[t] .. task_off[t+1]-1 and all s_* arrays are indexed by slot.

@@ -150,9 +150,11 @@ __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks
 //   order is (cost, pred_lat, -acc, id) order.  Entries that meet the SLO all miss the
 //   accuracy, the best of them is the one with the highest accuracy (bestA); entries that
 //   meet the accuracy all miss the SLO, the best being the one with the lowest latency
-//   (bestB); an entry that misses both can only win with accuracy above bestA's, latency
-//   not above bestB's and a latency overshoot that alone stays below the best distance so
-//   far, so the walk in latency order stops early.
+//   (bestB); an entry that misses both can only win with accuracy above bestA's and latency
+//   not above bestB's, and then only if no other entry is at least as fast and at least as
+//   accurate (for slo > 0 such an entry is strictly closer), so only those "stair" entries
+//   are walked, in latency order, until the latency overshoot alone exceeds the best
+//   distance so far.  For slo = 0 the accuracy term vanishes: the answer is the fastest entry.
 //   List without index: walk it in global memory, for a feasible entry, then for the distance.
 template <class Img>
 __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t task,
@@ -166,7 +168,7 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
     const uint32_t F = sl.y & 0xFFu, Ks = (sl.y >> 8) & 0xFFu, Ka = sl.y >> 16;
     const SlowLayout SL = slow_layout(F, Ks, Ka);
     const uint32_t so = sl.x;
-    const uint4 h = img.v4(task * HDR_BYTES);
+    const uint4 h = img.v4(task * HDR_BYTES + ((threadIdx.x & 7u) << 4));   // this lane's copy
     const uint32_t t2 = (h.z & 0xFFFFu) << 2, width = (h.z >> 16) & 0xFFu;
     uint32_t r = 0;                                            // r = #{Pd <= slo}
 #pragma unroll
@@ -177,6 +179,7 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
     const uint32_t k = acc_rank(img, h.z, h.w, min_acc);
     const uint32_t pos = img.u8(t2 + r * width + k);
     if (pos < F) return img.u32(t2 - 4u - (pos << 2));
+    if (slo == 0u) return INFAAS_NO_FEASIBLE | img.u32(t2 - 4u - (img.v2(so + SL.bestB).y << 2));
     uint32_t acc_floor = 0;               // candidates that miss both need accuracy >= this
     uint32_t pred_cap = 0xFFFFFFFFu;      // ... and latency <= this
     if (r > 0) {                          // some entry meets the SLO (and misses the accuracy)
@@ -191,7 +194,7 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
       if (d < best || (d == best && Bv.y < best_p)) { best = d; best_p = Bv.y; }
       pred_cap = Bv.x;
     }
-    for (uint32_t o = img.u8(so + SL.ordStart + r); o < F; ++o) {   // latencies above the SLO, ascending
+    for (uint32_t o = img.u8(so + SL.ordStart + r); o < sl.w; ++o) {   // stair entries above the SLO, ascending
       const uint2 e = img.v2(so + SL.walk + (o << 3));
       if (e.x > pred_cap) break;
       const unsigned long long over = (unsigned long long)(e.x - slo) * 10000ull;

@@ -170,8 +170,8 @@ constexpr uint32_t BITS_OF_2_POW_32 = 0x4F800000u;
 struct IndexScratch {          // shared memory used while building one task's index
   uint32_t pred[256], Pd[256], ids[256];
   uint16_t acc[256], Ad[256];
-  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256], bucket[256];
-  uint32_t ks, ka, base;
+  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256], bucket[256], on_stair[256];
+  uint32_t ks, ka, base, fs;
 };
 
 // Header of a task without index (also entry n_tasks): every query reads "none".
@@ -209,15 +209,21 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   // distinct values ...
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {            // uniform trip count
     const uint32_t p = p0 + (tid >> 3);
-    uint32_t dup = 0;                                  // bit 0: an earlier entry has this latency; bit 1: accuracy
+    // bit 0: an earlier entry has this latency; bit 1: this accuracy; bit 2: some entry is at
+    // least as fast and at least as accurate, and better in one of the two
+    uint32_t dup = 0;
     if (p < F) {
       const uint32_t pp = S.pred[p], pa = S.acc[p];
-      for (uint32_t q = sub; q < p; q += 8) dup |= (S.pred[q] == pp ? 1u : 0u) | (S.acc[q] == pa ? 2u : 0u);
+      for (uint32_t q = sub; q < F; q += 8) {
+        const uint32_t qp = S.pred[q], qa = S.acc[q];
+        if (q < p) dup |= (qp == pp ? 1u : 0u) | (qa == pa ? 2u : 0u);
+        dup |= (qp <= pp && qa >= pa && (qp < pp || qa > pa)) ? 4u : 0u;
+      }
     }
     dup = group8_or(dup);
-    if (p < F && sub == 0) { S.firstP[p] = !(dup & 1u); S.firstA[p] = !(dup & 2u); }
+    if (p < F && sub == 0) { S.firstP[p] = !(dup & 1u); S.firstA[p] = !(dup & 2u); S.on_stair[p] = !(dup & 4u); }
   }
-  if (tid == 0) { S.ks = 0; S.ka = 0; }
+  if (tid == 0) { S.ks = 0; S.ka = 0; S.fs = 0; }
   __syncthreads();
   // ... and their ranks
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {
@@ -237,10 +243,11 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
       S.Ad[ra] = S.acc[p];
       atomicMax(&S.ks, rp + 1);
       atomicMax(&S.ka, ra + 1);
+      if (S.on_stair[p]) atomicAdd(&S.fs, 1u);
     }
   }
   __syncthreads();
-  const uint32_t Ks = S.ks, Ka = S.ka;
+  const uint32_t Ks = S.ks, Ka = S.ka, Fs = S.fs;
   // SLO buckets: they cover the list's latencies up to the largest SLO asked for so far (as a
   // bit mask: every SLO seen is <= cap); larger latencies share bucket 255
   uint32_t cap = *c.slo_seen | SLO_CAP_FLOOR_US;
@@ -341,7 +348,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     uint32_t best = 0xFFu, best_acc = 0, cnt = 0;               // highest accuracy among ranks < r
     for (uint32_t p = 0; p < F; ++p) {
       if (S.idxP[p] < r) {
-        ++cnt;
+        cnt += S.on_stair[p];
         if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
       }
     }
@@ -359,9 +366,11 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   // small copies, after the short loops above
   uint32_t *ids_end = reinterpret_cast<uint32_t *>(blk + BL.t2);   // ids, reversed; slot F holds PENDING
   share(3 * B / 4, B / 8, F + 1u, [&](uint32_t p) { ids_end[-1 - (int)p] = p < F ? S.ids[p] : PENDING; });
-  uint2 *walk = reinterpret_cast<uint2 *>(slow + SL.walk);
-  share(7 * B / 8, B / 16, F, [&](uint32_t o) {
-    const uint32_t p = S.order[o];
+  uint2 *walk = reinterpret_cast<uint2 *>(slow + SL.walk);      // the stair entries, ascending latency
+  share(7 * B / 8, B / 16, F, [&](uint32_t p) {
+    if (!S.on_stair[p]) return;
+    uint32_t o = 0;                                             // stair entries have distinct latencies
+    for (uint32_t q = 0; q < F; ++q) o += S.on_stair[q] && S.pred[q] < S.pred[p];
     walk[o] = make_uint2(S.pred[p], (uint32_t)S.acc[p] | (p << 16));
   });
   uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
@@ -370,7 +379,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   const uint32_t cb = ((base + BL.bitmap) >> 2) - acc_lo / ACC_WORD_BITS;
   write_header(c, t, make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
                                 ((base + BL.t2) >> 2) | (width << 16) | (nbw << 24), acc_lo | (cb << 16)));
-  if (tid == 0) c.slow[t] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, 0u);
+  if (tid == 0) c.slow[t] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs);
   return true;
 }
 
