@@ -43,7 +43,8 @@ namespace infaas {
 //   dummy  64 bytes (what tasks without an index point at: every query of theirs reads
 //          "none" and goes to the slow path)
 //   var    per-task blocks, each 64-byte aligned:
-//          ids   u32[F + 1] in REVERSE order: ids[p] sits at t2_off - 4 - 4p, and the slot
+//          ids   u32[F + 1] in REVERSE order: ids[p] sits at t2_off - 4 - 4p (t2_off is a
+//                multiple of 16), and the slot
 //                of p = F holds PENDING -- the fast path needs no compare for "none"
 //          T2    u8[(Ks + 2) * (Ka + 1)]  at t2_off
 //          bitmap u32[nbw]
@@ -51,11 +52,11 @@ namespace infaas {
 //
 // Header words:
 //   w0 = float 2^-S          w1 = float -bmin
-//   w2 = t2_off / 4 | (Ka + 1) << 16 | nbw << 24
+//   w2 = t2_off / 16 | (Ka + 1) << 16 | nbw << 24
 //   w3 = acc_lo | cb << 16    acc_lo = multiple of 24 at or below the smallest accuracy,
-//                             cb = bitmap_off / 4 - acc_lo / 24 (word w of the bitmap, for
-//                             an accuracy a clamped to [acc_lo, acc_lo + 24 nbw - 1], is
-//                             word cb + a / 24 of the image)
+//                             cb = (bitmap_off - t2_off) / 4 + CB_BIAS - acc_lo / 24 (the bitmap
+//                             word for an accuracy a clamped to [acc_lo, acc_lo + 24 nbw - 1]
+//                             is word cb - CB_BIAS + a / 24 counted from t2_off)
 //
 // Per task in global memory (`regions`): keys u64[V] (pred_lat | acc_bp << 32, scan order,
 // F used) and ids u32[V], for lists without an index and for inspection.
@@ -65,7 +66,8 @@ constexpr uint32_t SLO_BUCKETS = 256;
 constexpr uint32_t ACC_WORD_BITS = 24;
 constexpr uint32_t MAX_ACC_WORDS = 255;          // nbw is an 8-bit field: 6120 basis points
 constexpr uint32_t HDR_BYTES = 128;              // 8 copies x 16 bytes
-constexpr uint32_t IMAGE_WORD_LIMIT = 1u << 16;  // t2_off / 4 and cb are 16-bit fields
+constexpr uint32_t IMAGE_T2_LIMIT = 1u << 20;    // t2_off / 16 is a 16-bit field
+constexpr uint32_t CB_BIAS = 512;                // keeps the header's bitmap field non-negative
 constexpr uint32_t SLO_CAP_FLOOR_US = (1u << 20) - 1u;  // the buckets cover latencies at least up to here
 constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-2)
 
@@ -111,7 +113,7 @@ struct BlockLayout {
 };
 inline __host__ __device__ BlockLayout block_layout(uint32_t F, uint32_t Ks, uint32_t Ka, uint32_t nbw) {
   BlockLayout B;
-  B.t2 = 4u * (F + 1u);
+  B.t2 = round_up_u32(4u * (F + 1u), 16u);
   B.bitmap = round_up_u32(B.t2 + (Ks + 2u) * (Ka + 1u), 4u);
   B.slow = round_up_u32(B.bitmap + 4u * nbw, 8u);
   B.bytes = round_up_u32(B.slow + slow_layout(F, Ks, Ka).bytes, 64u);

@@ -110,13 +110,14 @@ struct GlobalImage {
 __device__ __forceinline__ uint32_t div24(uint32_t a) { return __umulhi(a, 178956971u); }
 
 // k = #{distinct list accuracies < min_acc} from the bitmap with running popcounts.
-// w2, w3: header words (see common.cuh).
+// w2, w3: header words (see common.cuh); t2: image offset of the task's T2.
 template <class Img>
-__device__ __forceinline__ uint32_t acc_rank(const Img &img, uint32_t w2, uint32_t w3, uint32_t min_acc) {
+__device__ __forceinline__ uint32_t acc_rank(const Img &img, uint32_t w2, uint32_t w3, uint32_t t2,
+                                             uint32_t min_acc) {
   const uint32_t acc_lo = w3 & 0xFFFFu, cb = __umulhi(w3, 1u << 16), nbw = __umulhi(w2, 1u << 8);
   const uint32_t a = min(max(min_acc, acc_lo), acc_lo + ACC_WORD_BITS * nbw - 1u);
   const uint32_t w = div24(a);
-  const uint32_t word = img.u32((cb + w) << 2);
+  const uint32_t word = img.u32(t2 - 4u * CB_BIAS + ((cb + w) << 2));
   const uint32_t below = word & ((1u << (a - w * ACC_WORD_BITS)) - 1u);   // prefix byte masked off: shift < 24
   return __umulhi(word, 1u << 8) + __popc(below);
 }
@@ -137,8 +138,8 @@ __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks
   asm("cvt.rmi.sat.u8.f32 %0, %1;" : "=r"(j) : "f"(fmaf(code, __uint_as_float(h.x), __uint_as_float(h.y))));
   const uint32_t rec = img.u32(rec_off + t * (4u * SLO_BUCKETS) + (j << 2));
   const uint32_t r = __umulhi(rec + (slo & 0x00FFFFFFu), 1u << 8);
-  const uint32_t k = acc_rank(img, h.z, h.w, min_acc);
-  const uint32_t t2 = (h.z & 0xFFFFu) << 2, width = (h.z >> 16) & 0xFFu;
+  const uint32_t t2 = (h.z & 0xFFFFu) << 4, width = (h.z >> 16) & 0xFFu;
+  const uint32_t k = acc_rank(img, h.z, h.w, t2, min_acc);
   const uint32_t pos = img.u8(t2 + r * width + k);
   return img.u32(t2 - 4u - (pos << 2));
 }
@@ -169,14 +170,14 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
     const SlowLayout SL = slow_layout(F, Ks, Ka);
     const uint32_t so = sl.x;
     const uint4 h = img.v4(task * HDR_BYTES + ((threadIdx.x & 7u) << 4));   // this lane's copy
-    const uint32_t t2 = (h.z & 0xFFFFu) << 2, width = (h.z >> 16) & 0xFFu;
+    const uint32_t t2 = (h.z & 0xFFFFu) << 4, width = (h.z >> 16) & 0xFFu;
     uint32_t r = 0;                                            // r = #{Pd <= slo}
 #pragma unroll
     for (uint32_t step = 128; step; step >>= 1) {
       const uint32_t probe = r + step;
       if (probe <= Ks && img.u32(so + SL.Pd + ((probe - 1u) << 2)) <= slo) r = probe;
     }
-    const uint32_t k = acc_rank(img, h.z, h.w, min_acc);
+    const uint32_t k = acc_rank(img, h.z, h.w, t2, min_acc);
     const uint32_t pos = img.u8(t2 + r * width + k);
     if (pos < F) return img.u32(t2 - 4u - (pos << 2));
     if (slo == 0u) return INFAAS_NO_FEASIBLE | img.u32(t2 - 4u - (img.v2(so + SL.bestB).y << 2));

@@ -74,30 +74,36 @@ tally_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_varia
 
 // Same tallies with a private histogram per CTA in shared memory (one u32 bin per variant):
 // shared-memory atomics absorb the hot variants, and each CTA adds only its non-zero bins
-// to the global counts at the end.  Used when the bins fit and the batch is large.
+// to the global counts at the end.  Used when the batch is large.  If the bins of all
+// variants do not fit, the ids are split into `parts` ranges of `bins` ids: CTA b counts
+// range b % parts over the share b / parts of the decisions (every range sees all
+// decisions); the counters come from range 0 alone.
 constexpr int TALLY_SMEM_THREADS = 512;
 
 __global__ void __launch_bounds__(TALLY_SMEM_THREADS)
-tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_variants,
-                  uint32_t *__restrict__ count_by_id, unsigned long long *__restrict__ counters) {
+tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_variants, uint32_t bins,
+                  uint32_t parts, uint32_t *__restrict__ count_by_id,
+                  unsigned long long *__restrict__ counters) {
   extern __shared__ uint32_t hist[];
   __shared__ uint32_t blk[3];
-  for (uint32_t i = threadIdx.x; i < n_variants; i += blockDim.x) hist[i] = 0;
+  const uint32_t part = blockIdx.x % parts, lo = part * bins, share = blockIdx.x / parts;
+  const uint32_t my_bins = min(bins, n_variants - lo);
+  for (uint32_t i = threadIdx.x; i < my_bins; i += blockDim.x) hist[i] = 0;
   if (threadIdx.x < 3) blk[threadIdx.x] = 0;
   __syncthreads();
   // per decision: one compare + predicated shared-memory atomic, and two counters; invalid
   // decisions are what remains of the total
   uint32_t n_feas = 0, n_nofeas = 0, n_seen = 0;
   auto one = [&](uint32_t d) {
-    if (d < n_variants) atomicAdd(&hist[d], 1u);                 // d < n_variants < 2^31: bit 31 clear
-    n_feas += d < n_variants;
+    if (d - lo < my_bins) atomicAdd(&hist[d - lo], 1u);         // unsigned: ids below lo wrap around
+    n_feas += d < n_variants;                                    // d < n_variants < 2^31: bit 31 clear
     n_nofeas += (d - INFAAS_NO_FEASIBLE) < 0x7FFFFFFFu;          // bit 31 set and not INFAAS_INVALID
   };
   const uint32_t n4 = (uint32_t)(n >> 2);                        // n <= 2^32 - 1 (checked by the caller)
-  const uint32_t stride = gridDim.x * blockDim.x;
+  const uint32_t stride = (gridDim.x / parts) * blockDim.x;
   const uint4 *dec4 = reinterpret_cast<const uint4 *>(decision);
   // four 128-bit loads in flight per thread
-  uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  uint32_t i = share * blockDim.x + threadIdx.x;
   for (; n4 >= 3 * stride && i < n4 - 3 * stride; i += 4 * stride) {
     const uint4 d0 = __ldcs(dec4 + i), d1 = __ldcs(dec4 + i + stride);
     const uint4 d2 = __ldcs(dec4 + i + 2 * stride), d3 = __ldcs(dec4 + i + 3 * stride);
@@ -112,20 +118,20 @@ tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_
     one(d.x); one(d.y); one(d.z); one(d.w);
     n_seen += 4;
   }
-  if (blockIdx.x == 0 && threadIdx.x < (n & 3)) { one(decision[((uint64_t)n4 << 2) + threadIdx.x]); ++n_seen; }
+  if (share == 0 && threadIdx.x < (n & 3)) { one(decision[((uint64_t)n4 << 2) + threadIdx.x]); ++n_seen; }
   uint32_t n_inval = n_seen - n_feas - n_nofeas;
   n_feas = __reduce_add_sync(0xFFFFFFFFu, n_feas);
   n_nofeas = __reduce_add_sync(0xFFFFFFFFu, n_nofeas);
   n_inval = __reduce_add_sync(0xFFFFFFFFu, n_inval);
-  if ((threadIdx.x & 31) == 0) {
+  if ((threadIdx.x & 31) == 0 && part == 0) {
     atomicAdd(&blk[0], n_feas);
     atomicAdd(&blk[1], n_nofeas);
     atomicAdd(&blk[2], n_inval);
   }
   __syncthreads();
-  for (uint32_t i = threadIdx.x; i < n_variants; i += blockDim.x) {
+  for (uint32_t i = threadIdx.x; i < my_bins; i += blockDim.x) {
     const uint32_t h = hist[i];
-    if (h) atomicAdd(&count_by_id[i], h);
+    if (h) atomicAdd(&count_by_id[lo + i], h);
   }
   if (threadIdx.x < 3 && blk[threadIdx.x]) atomicAdd(&counters[threadIdx.x], (unsigned long long)blk[threadIdx.x]);
 }
@@ -177,7 +183,9 @@ struct IndexScratch {          // shared memory used while building one task's i
 // Header of a task without index (also entry n_tasks): every query reads "none".
 __device__ __forceinline__ uint4 dummy_header(uint32_t n_tasks) {
   const uint32_t dummy = image_dummy_offset(n_tasks);
-  return make_uint4(0u, 0u, ((dummy + 4u) >> 2) | (0u << 16) | (1u << 24), 0u | (((dummy + 8u) >> 2) << 16));
+  // T2 (one byte, 0) at dummy + 16, the id slot of position 0 (PENDING) just below it, the bitmap
+  // (one word, 0) at dummy + 32
+  return make_uint4(0u, 0u, ((dummy + 16u) >> 4) | (0u << 16) | (1u << 24), 0u | ((4u + CB_BIAS) << 16));
 }
 __device__ __forceinline__ void write_header(const DeviceCatalog &c, uint32_t t, uint4 h) {
   if (threadIdx.x < HDR_BYTES / 16u) reinterpret_cast<uint4 *>(c.image + HDR_BYTES * t)[threadIdx.x] = h;
@@ -281,7 +289,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     uint32_t base = 0xFFFFFFFFu;
     if (nbw <= MAX_ACC_WORDS) {
       base = image_var_offset(c.n_tasks) + atomicAdd(&c.rebuild_ctr[1], BL.bytes);
-      if (base + BL.bytes > c.image_capacity || ((base + BL.bitmap) >> 2) >= IMAGE_WORD_LIMIT) base = 0xFFFFFFFFu;
+      if (base + BL.bytes > c.image_capacity || base + BL.t2 >= IMAGE_T2_LIMIT) base = 0xFFFFFFFFu;
     }
     S.base = base;
   }
@@ -376,9 +384,9 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
   share(15 * B / 16, B / 16, Ks, [&](uint32_t i) { Pd_g[i] = S.Pd[i]; });
 
-  const uint32_t cb = ((base + BL.bitmap) >> 2) - acc_lo / ACC_WORD_BITS;
+  const uint32_t cb = ((BL.bitmap - BL.t2) >> 2) + CB_BIAS - acc_lo / ACC_WORD_BITS;
   write_header(c, t, make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
-                                ((base + BL.t2) >> 2) | (width << 16) | (nbw << 24), acc_lo | (cb << 16)));
+                                ((base + BL.t2) >> 4) | (width << 16) | (nbw << 24), acc_lo | (cb << 16)));
   if (tid == 0) c.slow[t] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs);
   return true;
 }
@@ -547,7 +555,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     write_header(c, T, dummy_header(T));
     uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T)) + T * SLO_BUCKETS;
     for (uint32_t j = tid; j < SLO_BUCKETS; j += B) rec[j] = 0u;
-    if (tid < 16) reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid == 0 ? PENDING : 0u;
+    if (tid < 16) reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid == 3 ? PENDING : 0u;
   }
   if (tid == 0) {
     c.f_len[t] = F;
@@ -577,20 +585,23 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
 }  // namespace
 
 constexpr uint32_t TALLY_SMEM_MAX_VARIANTS = 49152;   // 192 KB of bins
+constexpr uint32_t TALLY_SMEM_MAX_PARTS = 8;           // beyond this many id ranges: global atomics
 constexpr uint64_t TALLY_SMEM_MIN_N = 1u << 18;        // below this the zero/flush passes cost more than they save
 
 cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uint64_t n,
                          cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
-  if (n >= TALLY_SMEM_MIN_N && c.n_variants <= TALLY_SMEM_MAX_VARIANTS) {
-    const size_t smem = (size_t)c.n_variants * 4;
+  const uint32_t parts = (c.n_variants + TALLY_SMEM_MAX_VARIANTS - 1) / TALLY_SMEM_MAX_VARIANTS;
+  if (n >= TALLY_SMEM_MIN_N && parts <= TALLY_SMEM_MAX_PARTS) {
+    const uint32_t bins = ((c.n_variants + parts - 1) / parts + 3u) & ~3u;
+    const size_t smem = (size_t)bins * 4;
     const uint32_t per_sm = smem > 100 * 1024 ? 1 : 2;
     uint64_t want = ((n >> 2) + TALLY_SMEM_THREADS * 8 - 1) / (TALLY_SMEM_THREADS * 8);
-    uint64_t grid = (uint64_t)148 * per_sm;
-    if (grid > want) grid = want;
-    if (grid < 1) grid = 1;
-    tally_smem_kernel<<<(uint32_t)grid, TALLY_SMEM_THREADS, smem, stream>>>(
-        d_decision, n, c.n_variants, c.count_by_id, c.counters);
+    uint64_t shares = (uint64_t)148 * per_sm / parts;          // CTAs per id range
+    if (shares > want) shares = want;
+    if (shares < 1) shares = 1;
+    tally_smem_kernel<<<(uint32_t)(shares * parts), TALLY_SMEM_THREADS, smem, stream>>>(
+        d_decision, n, c.n_variants, bins, parts, c.count_by_id, c.counters);
     return cudaGetLastError();
   }
   uint64_t want = ((n >> 2) + 255) / 256;

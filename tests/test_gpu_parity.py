@@ -325,3 +325,22 @@ def test_split_update_with_summed_counts_matches_whole_window():
     finally:
         for cat in cats:
             cat.free()
+
+
+def test_large_batch_over_a_catalog_whose_tally_bins_need_two_ranges():
+    """65,536 variants: the shared-memory tally splits the ids into two ranges; 2M queries in
+    one launch (image read from global memory: it does not fit in shared memory)."""
+    import paper_1905_13348_b200 as P
+    w = W.make("C5", n_windows=32)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    try:
+        for rnd in range(2):
+            want = o.select(w.task, w.slo_us, w.min_acc_bp, _threads())
+            d_dec = gpu_select(cat, w.task, w.slo_us, w.min_acc_bp)
+            assert np.array_equal(_to_host_u32(d_dec), want), rnd
+            P.infaas_load_update(cat, d_dec, 32 * w.window_us)
+            o.load_update(want, 32 * w.window_us)
+            _assert_state_fast(cat, o, w.rows)
+    finally:
+        cat.free()
