@@ -57,16 +57,16 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Re-reads the image size from the device and sizes the selection kernel's shared memory
-// with headroom for growth between two such refreshes.
+// Re-reads the image size from the device and decides how much shared memory the selection
+// kernel asks for: all of it while the image fits (it may grow or shrink between two such
+// refreshes without a change of plan), none for the image if it does not -- the kernel
+// then reads it from global memory and the space is worth more as L1 cache.
 int refresh_select_plan(infaas_catalog *c, cudaStream_t stream) {
   uint32_t hdr[4] = {0, 0, 0, 0};
   CUDA_TRY(cudaMemcpyAsync(hdr, c->d.image_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, stream));
   CUDA_TRY(cudaStreamSynchronize(stream));
-  uint64_t want = (uint64_t)hdr[0] + hdr[0] / 2 + 4096;
-  if (want > c->worst_image_bytes) want = c->worst_image_bytes;
-  if (want > infaas::SELECT_MAX_SMEM) want = infaas::SELECT_MAX_SMEM;   // the launcher trims further
-  c->select_smem = (uint32_t)((want + 15) & ~(uint64_t)15);
+  const uint32_t room = infaas::select_image_smem(infaas::SELECT_MAX_SMEM);
+  c->select_smem = hdr[0] <= room ? room : 0u;
   return INFAAS_OK;
 }
 
