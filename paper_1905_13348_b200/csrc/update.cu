@@ -88,14 +88,17 @@ tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_
   __shared__ uint32_t blk[3];
   const uint32_t part = blockIdx.x % parts, lo = part * bins, share = blockIdx.x / parts;
   const uint32_t my_bins = min(bins, n_variants - lo);
+  const uint32_t spare = my_bins + (threadIdx.x & 31u);
   for (uint32_t i = threadIdx.x; i < my_bins; i += blockDim.x) hist[i] = 0;
   if (threadIdx.x < 3) blk[threadIdx.x] = 0;
   __syncthreads();
-  // per decision: one compare + predicated shared-memory atomic, and two counters; invalid
+  // per decision: one shared-memory atomic and two counters; invalid
   // decisions are what remains of the total
   uint32_t n_feas = 0, n_nofeas = 0, n_seen = 0;
   auto one = [&](uint32_t d) {
-    if (d - lo < my_bins) atomicAdd(&hist[d - lo], 1u);         // unsigned: ids below lo wrap around
+    // no branch: what is not in this CTA's range (ids below lo wrap around) lands in one of 32
+    // spare bins, one per lane, that nobody reads
+    atomicAdd(&hist[min(d - lo, spare)], 1u);
     n_feas += d < n_variants;                                    // d < n_variants < 2^31: bit 31 clear
     n_nofeas += (d - INFAAS_NO_FEASIBLE) < 0x7FFFFFFFu;          // bit 31 set and not INFAAS_INVALID
   };
@@ -594,7 +597,7 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
   const uint32_t parts = (c.n_variants + TALLY_SMEM_MAX_VARIANTS - 1) / TALLY_SMEM_MAX_VARIANTS;
   if (n >= TALLY_SMEM_MIN_N && parts <= TALLY_SMEM_MAX_PARTS) {
     const uint32_t bins = ((c.n_variants + parts - 1) / parts + 3u) & ~3u;
-    const size_t smem = (size_t)bins * 4;
+    const size_t smem = (size_t)(bins + 32) * 4;                 // 32 spare bins
     const uint32_t per_sm = smem > 100 * 1024 ? 1 : 2;
     uint64_t want = ((n >> 2) + TALLY_SMEM_THREADS * 8 - 1) / (TALLY_SMEM_THREADS * 8);
     uint64_t shares = (uint64_t)148 * per_sm / parts;          // CTAs per id range
@@ -612,7 +615,7 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
 
 cudaError_t prepare_rebuild_kernel() {
   cudaError_t e = cudaFuncSetAttribute(tally_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)(TALLY_SMEM_MAX_VARIANTS * 4));
+                                       (int)((TALLY_SMEM_MAX_VARIANTS + 32) * 4));
   if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(rebuild_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)REBUILD_MAX_SMEM);
