@@ -179,7 +179,8 @@ constexpr uint32_t BITS_OF_2_POW_32 = 0x4F800000u;
 struct IndexScratch {          // shared memory used while building one task's index
   uint32_t pred[256], Pd[256], ids[256];
   uint16_t acc[256], Ad[256];
-  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], order[256], bucket[256], on_stair[256];
+  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], bucket[256], on_stair[256];
+  unsigned long long Lmask[256][4], Amask[256][4];   // positions by latency rank < r / accuracy rank >= k
   uint32_t ks, ka, base, fs;
 };
 
@@ -270,16 +271,19 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   const uint32_t bmin = clo >> sh, Sh = 16u + sh;
   for (uint32_t i = tid; i < Ks; i += B)
     S.bucket[i] = (unsigned char)(min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1));
-  // positions ordered by rank of pred_lat (ties in scan order)
-  for (uint32_t p0 = 0; p0 < F; p0 += PB) {
-    const uint32_t p = p0 + (tid >> 3);
-    uint32_t o = 0;
-    if (p < F) {
-      const uint32_t ip = S.idxP[p];
-      for (uint32_t q = sub; q < F; q += 8) o += S.idxP[q] < ip || (S.idxP[q] == ip && q < p);
+  // position masks: Lmask[r] = positions whose latency rank is < r, Amask[k] = positions whose
+  // accuracy rank is >= k (64 positions per word); T2[r][k] is the first bit of their intersection
+  const uint32_t nw = (F + 63u) >> 6;
+  for (uint32_t x = tid; x < 2u * 256u * nw; x += B) {
+    const uint32_t which = x / (256u * nw), y = x - which * 256u * nw, rk = y / nw, w = y - rk * nw;
+    if (rk > (which ? Ka : Ks)) continue;
+    unsigned long long m = 0;
+    const uint32_t p1 = min(F, 64u * w + 64u);
+    for (uint32_t p = 64u * w; p < p1; ++p) {
+      const bool in = which ? S.idxA[p] >= rk : S.idxP[p] < rk;
+      m |= (unsigned long long)in << (p & 63u);
     }
-    o = group8_add(o);
-    if (p < F && sub == 0) S.order[o] = (unsigned char)p;
+    (which ? S.Amask : S.Lmask)[rk][w] = m;
   }
 
   // block layout and its place in the image
@@ -315,8 +319,10 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     const uint32_t r = cell / width, k = cell - r * width;
     uint32_t pos = F;
     if (r >= 1 && r <= Ks)
-      for (uint32_t p = 0; p < F; ++p)
-        if (S.idxP[p] < r && S.idxA[p] >= k) { pos = p; break; }
+      for (uint32_t w = 0; w < nw; ++w) {
+        const unsigned long long m = S.Lmask[r][w] & S.Amask[k][w];
+        if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
+      }
     T2[cell] = (unsigned char)pos;
   });
 
@@ -447,37 +453,28 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   __syncthreads();
 
   uint32_t my_kept = 0;
-  if (sort_n <= RANK_SORT_MAX) {
-    // 2+3 (small tasks).  Rank sort fused with the prune: entry q sorts before p iff its key
-    // (cost, pred, 10000-acc, local index) is smaller, and it dominates p iff in addition
-    // pred_q <= pred_p and acc_q >= acc_p (its cost is not larger by the key order, and it
-    // differs in some attribute or has the smaller id).  G lanes share an entry's comparisons.
-    unsigned long long *o64 = reinterpret_cast<unsigned long long *>(keep + sort_n + ((8u - ((13u * sort_n) & 7u)) & 7u));
-    uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);
+  const bool small = sort_n <= RANK_SORT_MAX;
+  unsigned long long *o64 = reinterpret_cast<unsigned long long *>(keep + sort_n + ((8u - ((13u * sort_n) & 7u)) & 7u));
+  uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);   // (only there for small tasks)
+  if (small) {
+    // 3 (small tasks, before any sort).  q dominates p iff cost_q <= cost_p, pred_q <= pred_p,
+    // acc_q >= acc_p and it differs in some attribute or has the smaller id -- which, given
+    // the three inequalities, is the same as its key (cost, pred, 10000-acc, local index)
+    // being smaller.  G lanes share an entry's comparisons.
     const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
-    uint32_t rank = 0, dom = 0;
-    unsigned long long a64 = 0;
-    uint32_t a32 = 0;
+    uint32_t dom = 0;
     if (p < V) {
-      a64 = k64[p]; a32 = k32[p];
-      const uint32_t pred_p = (uint32_t)a64, inv_p = a32 >> 16;
+      const unsigned long long a64 = k64[p];
+      const uint32_t a32 = k32[p], cost_p = (uint32_t)(a64 >> 32), pred_p = (uint32_t)a64, inv_p = a32 >> 16;
       for (uint32_t q = sidx; q < V; q += G) {
         const unsigned long long b64 = k64[q];
         const uint32_t b32 = k32[q];
-        const bool less = key_less(b64, b32, a64, a32);
-        rank += less;
-        dom |= (less && (uint32_t)b64 <= pred_p && (b32 >> 16) <= inv_p) ? 1u : 0u;
+        dom |= ((uint32_t)(b64 >> 32) <= cost_p && (uint32_t)b64 <= pred_p && (b32 >> 16) <= inv_p &&
+                key_less(b64, b32, a64, a32)) ? 1u : 0u;
       }
     }
-    for (uint32_t o = G >> 1; o; o >>= 1) {            // G is a power of two, groups are lane-aligned
-      rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
-      dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);
-    }
-    if (p < V && sidx == 0) {
-      o64[rank] = a64; o32[rank] = a32; keep[rank] = !dom;
-      my_kept = !dom;
-    }
-    k64 = o64; k32 = o32;
+    for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
+    if (p < V && sidx == 0) { keep[p] = !dom; my_kept = !dom; }
   } else {
     // 2. bitonic sort of P keys, ascending in (cost, pred, 10000-acc, local index)
     for (uint32_t k = 2; k <= P; k <<= 1) {
@@ -528,6 +525,13 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   // 4. compact into the task's region (scan order): keys and ids
   unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(region);
   uint32_t *ids_g = reinterpret_cast<uint32_t *>(region + 8u * V);
+  auto emit = [&](uint32_t pos, unsigned long long v64, uint32_t v32) {   // list position pos
+    const uint32_t pred_p = (uint32_t)v64, acc = 10000u - (v32 >> 16);
+    const uint32_t id = c.s_id[base + (v32 & 0xFFFFu)];
+    keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
+    ids_g[pos] = id;
+    if (indexed) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }
+  };
   uint32_t kept_so_far = 0;
   for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
     const uint32_t p = p0 + tid;
@@ -535,15 +539,28 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     uint32_t total;
     const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
     if (kp) {
-      const uint32_t pred_p = (uint32_t)k64[p], acc = 10000u - (k32[p] >> 16);
-      const uint32_t id = c.s_id[base + (k32[p] & 0xFFFFu)];
-      keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
-      ids_g[pos] = id;
-      if (indexed) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }
+      if (small) { o64[pos] = k64[p]; o32[pos] = k32[p]; }      // survivors, not yet in order
+      else emit(pos, k64[p], k32[p]);
     }
     kept_so_far += total;
   }
   __syncthreads();
+  if (small) {
+    // 2 (small tasks): the survivors' list positions by counting smaller keys
+    uint32_t PF = 1;
+    while (PF < F) PF <<= 1;
+    const uint32_t G = min(32u, B / PF), i = tid / G, sidx = tid % G;
+    uint32_t rank = 0;
+    unsigned long long a64 = 0;
+    uint32_t a32 = 0;
+    if (i < F) {
+      a64 = o64[i]; a32 = o32[i];
+      for (uint32_t j = sidx; j < F; j += G) rank += key_less(o64[j], o32[j], a64, a32);
+    }
+    for (uint32_t o = G >> 1; o; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+    if (i < F && sidx == 0) emit(rank, a64, a32);
+    __syncthreads();
+  }
   if (indexed) indexed = build_index(c, t, F, S);
   if (!indexed) {
     // no index: header and records that make every query of this task read "none"
