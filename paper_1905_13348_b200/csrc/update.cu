@@ -421,6 +421,13 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint32_t P = 1;
   while (P < V) P <<= 1;
 
+  // small tasks have, behind the sort buffers, a second copy of the keys (survivors of the
+  // prune) and the attributes packed for the prune
+  const bool small = sort_n <= RANK_SORT_MAX;
+  unsigned long long *o64 = reinterpret_cast<unsigned long long *>(keep + sort_n + ((16u - ((13u * sort_n) & 15u)) & 15u));
+  uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);
+  uint4 *attr = reinterpret_cast<uint4 *>((reinterpret_cast<uintptr_t>(o32 + sort_n) + 15u) & ~(uintptr_t)15u);
+
   // 1. queue recursion, predicted latency, sort keys
   for (uint32_t i = tid; i < P; i += B) {
     if (i < V) {
@@ -443,8 +450,10 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       unsigned long long p = (unsigned long long)lat + (unsigned long long)queued * lat / batch;
       const uint32_t pred = p > U32_MAX_ ? U32_MAX_ : (uint32_t)p;
       c.s_pred[slot] = pred;
-      k64[i] = ((unsigned long long)c.s_cost[slot] << 32) | pred;
-      k32[i] = ((10000u - c.s_acc[slot]) << 16) | i;
+      const uint32_t cost = c.s_cost[slot], inv = 10000u - c.s_acc[slot];
+      k64[i] = ((unsigned long long)cost << 32) | pred;
+      k32[i] = (inv << 16) | i;
+      if (small) attr[i] = make_uint4(cost, pred, inv, i);
     } else {
       k64[i] = ~0ull;
       k32[i] = ~0u;
@@ -453,9 +462,6 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   __syncthreads();
 
   uint32_t my_kept = 0;
-  const bool small = sort_n <= RANK_SORT_MAX;
-  unsigned long long *o64 = reinterpret_cast<unsigned long long *>(keep + sort_n + ((8u - ((13u * sort_n) & 7u)) & 7u));
-  uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);   // (only there for small tasks)
   if (small) {
     // 3 (small tasks, before any sort).  q dominates p iff cost_q <= cost_p, pred_q <= pred_p,
     // acc_q >= acc_p and it differs in some attribute or has the smaller id -- which, given
@@ -464,13 +470,11 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
     uint32_t dom = 0;
     if (p < V) {
-      const unsigned long long a64 = k64[p];
-      const uint32_t a32 = k32[p], cost_p = (uint32_t)(a64 >> 32), pred_p = (uint32_t)a64, inv_p = a32 >> 16;
+      const uint4 a = attr[p];
       for (uint32_t q = sidx; q < V; q += G) {
-        const unsigned long long b64 = k64[q];
-        const uint32_t b32 = k32[q];
-        dom |= ((uint32_t)(b64 >> 32) <= cost_p && (uint32_t)b64 <= pred_p && (b32 >> 16) <= inv_p &&
-                key_less(b64, b32, a64, a32)) ? 1u : 0u;
+        const uint4 b = attr[q];                       // (cost, pred, 10000 - acc, local index)
+        if (b.x <= a.x && b.y <= a.y && b.z <= a.z)    // rare
+          dom |= (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w) ? 1u : 0u;
       }
     }
     for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
@@ -642,8 +646,8 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream) {
   uint32_t P = 1;
   while (P < c.max_task_variants) P <<= 1;
-  // small tasks: room for the rank sort's second copy of the keys (12 bytes per entry, 8-byte aligned)
-  size_t smem = (size_t)P * 13 + (P <= RANK_SORT_MAX ? (size_t)P * 12 + 8 : 0);
+  // small tasks: room for a second copy of the keys (12 bytes per entry) and the packed attributes (16)
+  size_t smem = (size_t)P * 13 + (P <= RANK_SORT_MAX ? (size_t)P * 28 + 32 : 0);
   rebuild_kernel<<<c.n_tasks, REBUILD_THREADS, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
   return cudaGetLastError();
 }
