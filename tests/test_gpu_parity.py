@@ -344,3 +344,42 @@ def test_large_batch_over_a_catalog_whose_tally_bins_need_two_ranges():
             _assert_state_fast(cat, o, w.rows)
     finally:
         cat.free()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_catalog_shapes(seed):
+    """Catalog shapes around the kernels' internal limits: task sizes on both sides of the
+    small-task sort limit and of the index limit, accuracy spans wider than the bitmap
+    supports, latencies from 1 us to beyond 2^24 us, many equal values, uneven load."""
+    rng = np.random.default_rng(1000 + seed)
+    sizes = rng.choice(np.array([1, 2, 3, 31, 32, 33, 200, 255, 256, 257, 511, 512, 513, 700, 1025]),
+                       size=int(rng.integers(3, 9)))
+    T = sizes.size + 1                               # the last task stays empty
+    task = np.repeat(np.arange(sizes.size), sizes)
+    nv = task.size
+    style = seed % 3
+    if style == 0:      # trade-off surface: long non-dominated lists, wide accuracy span
+        lat = np.exp(rng.uniform(np.log(1.0), np.log(3.0e7), nv))
+        cost = 1.0e6 / lat ** 0.5 * np.exp(0.3 * rng.standard_normal(nv))
+        acc = np.clip(10000 * (np.log(lat) / np.log(3.0e7)) + 300 * rng.standard_normal(nv), 0, 10000)
+    elif style == 1:    # few distinct values: ties everywhere
+        lat = rng.choice(np.array([1, 7, 100, 1000, 20000, 2**24, 2**24 + 1, 2**31]), nv).astype(float)
+        cost = rng.integers(1, 6, nv).astype(float)
+        acc = rng.choice(np.array([0, 1, 5000, 7000, 7001, 9999, 10000]), nv).astype(float)
+    else:               # independent attributes: short lists
+        lat = np.exp(rng.uniform(np.log(50.0), np.log(5.0e6), nv))
+        cost = rng.integers(1, 100000, nv).astype(float)
+        acc = rng.integers(5000, 9000, nv).astype(float)
+    rows = rows_from(task, rng.choice(np.array([1, 2, 8, 64, 65535]), nv),
+                     np.maximum(1, np.round(lat)).astype(np.uint64).clip(1, 2**32 - 1),
+                     np.round(acc).astype(np.int64), np.maximum(1, np.round(cost)).astype(np.uint64).clip(1, 2**32 - 1),
+                     rng.choice(np.array([0, 0, 0, 1, 5, 1000, 2**20]), nv))
+    rows = rows[rng.permutation(nv)]
+    n = 3 * 20011
+    q_task = rng.integers(0, T + 1, n).astype(np.uint16)
+    q_slo = np.where(rng.random(n) < 0.9, np.exp(rng.uniform(0, np.log(1.0e8), n)),
+                     rng.choice(np.array([0, 1, 2**24 - 1, 2**24, 2**32 - 1], dtype=np.float64), n)).astype(np.uint64)
+    q_slo = q_slo.clip(0, 2**32 - 1).astype(np.uint32)
+    q_acc = np.where(rng.random(n) < 0.9, rng.integers(0, 10001, n), rng.choice(np.array([0, 10001, 65535]), n)).astype(np.uint16)
+    w = W.Workload("shapes", T, rows, q_task, q_slo, q_acc, 20011, 50_000, "random shapes")
+    run_both(w)
