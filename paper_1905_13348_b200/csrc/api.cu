@@ -143,8 +143,18 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   if (scope.status != cudaSuccess) { delete c; return cuda_fail(scope.status); }
 
   // ---- one arena, carved into 256-byte aligned arrays ----
+  // lists longer than the index supports are cut into segments; every segment but a task's
+  // first needs a header and parameters outside the image
   uint64_t worst_image = infaas::image_var_offset(n_tasks);
-  for (uint32_t t = 0; t < n_tasks; ++t) worst_image += infaas::block_capacity(task_off[t + 1] - task_off[t]);
+  std::vector<uint32_t> seg_base(n_tasks + 1, 0);
+  for (uint32_t t = 0; t < n_tasks; ++t) {
+    const uint32_t V = task_off[t + 1] - task_off[t];
+    const uint32_t segs = V ? (V + infaas::INDEX_MAX_F - 1) / infaas::INDEX_MAX_F : 1;
+    seg_base[t + 1] = seg_base[t] + segs - 1;
+    worst_image += (uint64_t)(segs - 1) * infaas::block_capacity(infaas::INDEX_MAX_F) +
+                   infaas::block_capacity(V - (segs - 1) * infaas::INDEX_MAX_F);
+  }
+  const uint32_t n_extra = seg_base[n_tasks];
   if (worst_image > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
   size_t total = 0;
   auto carve = [&total](size_t bytes) { size_t off = total; total += round_up(bytes, 256); return off; };
@@ -155,7 +165,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
   const size_t o_regions = carve((size_t)region_bytes);
-  const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve((size_t)n_tasks * 16);
+  const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve(((size_t)n_tasks + n_extra) * 16);
+  const size_t o_seg_base = carve((n_tasks + 1) * 4), o_xhdr = carve((size_t)n_extra * 16 + 16);
   const size_t o_image = carve((size_t)worst_image), o_hdr = carve(16);
   const size_t o_counters = carve(24), o_rebuild = carve(32), o_err = carve(4), o_seen = carve(4);
 
@@ -173,6 +184,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   LOAD_TRY(cudaMemset(base, 0, total));
   LOAD_TRY(cudaMemcpy(base + o_task_off, task_off.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_reg_off, reg_off.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_seg_base, seg_base.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_lat, h_lat.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_batch, h_batch.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_acc, h_acc.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
@@ -198,6 +210,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.regions = base + o_regions;
   d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
   d.slow = reinterpret_cast<uint4 *>(base + o_slow);
+  d.seg_base = reinterpret_cast<const uint32_t *>(base + o_seg_base);
+  d.xhdr = reinterpret_cast<uint4 *>(base + o_xhdr);
   d.image = base + o_image;
   d.image_capacity = (uint32_t)worst_image;
   d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);

@@ -14,7 +14,10 @@ namespace infaas {
 // Scan list of a task: its non-dominated variants sorted by (cost, pred_lat, 10000-acc, id).
 // Position p in that order is what selection returns the smallest feasible of.
 //
-// For a list of F <= INDEX_MAX_F entries the rebuild kernel derives an exact index:
+// A list is cut into segments of at most INDEX_MAX_F consecutive positions (almost always
+// one).  The selection kernel's fast path looks at the first segment only; if that holds
+// nothing feasible the slow path goes through the others in order.  For a segment of F
+// entries the rebuild kernel derives an exact index:
 //   Pd[0..Ks)  distinct pred_lat values ascending,  Ad[0..Ka)  distinct acc_bp ascending,
 //   r(slo) = #{Pd <= slo},  k(min_acc) = #{Ad < min_acc},
 //   T2[r][k] = first position whose pred_lat is among the r smallest values and whose
@@ -126,8 +129,10 @@ inline __host__ __device__ uint32_t block_capacity(uint32_t V) {
 }
 inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_up_u32(12u * V, 64u); }
 
-// Slow-path parameters of a task (one uint4 per task, global memory).
-//   x = image offset of the slow tables   y = F | Ks << 8 | Ka << 16   z = flags   w = Fs
+// Slow-path parameters of a list segment (one uint4 each, global memory; a task's first
+// segment at index task, further segments at n_tasks + their index).
+//   x = image offset of the slow tables   y = F | Ks << 8 | Ka << 16   z = flags
+//   w = Fs | (1 + index of the task's next segment, 0 if none) << 8
 // ---------------------------------------------------------------------------------------
 // Device catalog.  "Slot" order: variants bucketed by task, ascending id inside a task;
 // task t owns slots task_off[t] .. task_off[t+1]-1 and all s_* arrays are indexed by slot.
@@ -151,7 +156,9 @@ struct DeviceCatalog {
 
   unsigned char *regions;    // per task: keys u64[V], ids u32[V] (scan order)
   uint32_t *f_len;           // [n_tasks] list length F
-  uint4 *slow;               // [n_tasks] slow-path parameters
+  uint4 *slow;               // [n_tasks + n_extra] slow-path parameters of the segments
+  const uint32_t *seg_base;  // [n_tasks + 1] index of each task's first further segment
+  uint4 *xhdr;               // [n_extra] headers of the further segments (first segments: in the image)
 
   unsigned char *image;      // packed image, image_capacity bytes, 256-byte aligned
   uint32_t image_capacity;

@@ -156,57 +156,88 @@ __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks
 //   accurate (for slo > 0 such an entry is strictly closer), so only those "stair" entries
 //   are walked, in latency order, until the latency overshoot alone exceeds the best
 //   distance so far.  For slo = 0 the accuracy term vanishes: the answer is the fastest entry.
+//   A list longer than INDEX_MAX_F is a chain of segments, each with tables of its own: the
+//   first segment with a feasible entry answers; otherwise the closest of the segments' misses.
 //   List without index: walk it in global memory, for a feasible entry, then for the distance.
+// One segment of a task's list (at most INDEX_MAX_F consecutive positions with their own
+// tables): returns the id of its first feasible entry, or PENDING after folding the
+// segment's nearest miss into (best, best_id); a later segment wins only with a strictly
+// smaller distance, since its positions are all higher.
 template <class Img>
-__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t task,
-                                                uint32_t slo, uint32_t min_acc) {
-  if (task >= c.n_tasks) return INFAAS_INVALID;
-  const uint4 sl = __ldg(c.slow + task);
-  if (sl.z & TASK_FLAG_INVALID) return INFAAS_INVALID;
-  unsigned long long best = ~0ull;
-  uint32_t best_p = 0;
-  if (!(sl.z & TASK_FLAG_NOT_INDEXED)) {
-    const uint32_t F = sl.y & 0xFFu, Ks = (sl.y >> 8) & 0xFFu, Ka = sl.y >> 16;
-    const SlowLayout SL = slow_layout(F, Ks, Ka);
-    const uint32_t so = sl.x;
-    const uint4 h = img.v4(task * HDR_BYTES + ((threadIdx.x & 7u) << 4));   // this lane's copy
-    const uint32_t t2 = (h.z & 0xFFFFu) << 4, width = (h.z >> 16) & 0xFFu;
-    uint32_t r = 0;                                            // r = #{Pd <= slo}
+__device__ __forceinline__ uint32_t slow_segment(const Img &img, const uint4 sl, const uint4 h, uint32_t slo,
+                                                 uint32_t min_acc, unsigned long long &best,
+                                                 uint32_t &best_id) {
+  const uint32_t F = sl.y & 0xFFu, Ks = (sl.y >> 8) & 0xFFu, Ka = sl.y >> 16, Fs = sl.w & 0xFFu;
+  const SlowLayout SL = slow_layout(F, Ks, Ka);
+  const uint32_t so = sl.x;
+  const uint32_t t2 = (h.z & 0xFFFFu) << 4, width = (h.z >> 16) & 0xFFu;
+  uint32_t r = 0;                                            // r = #{Pd <= slo}
 #pragma unroll
-    for (uint32_t step = 128; step; step >>= 1) {
-      const uint32_t probe = r + step;
-      if (probe <= Ks && img.u32(so + SL.Pd + ((probe - 1u) << 2)) <= slo) r = probe;
-    }
-    const uint32_t k = acc_rank(img, h.z, h.w, t2, min_acc);
-    const uint32_t pos = img.u8(t2 + r * width + k);
-    if (pos < F) return img.u32(t2 - 4u - (pos << 2));
-    if (slo == 0u) return INFAAS_NO_FEASIBLE | img.u32(t2 - 4u - (img.v2(so + SL.bestB).y << 2));
+  for (uint32_t step = 128; step; step >>= 1) {
+    const uint32_t probe = r + step;
+    if (probe <= Ks && img.u32(so + SL.Pd + ((probe - 1u) << 2)) <= slo) r = probe;
+  }
+  const uint32_t k = acc_rank(img, h.z, h.w, t2, min_acc);
+  const uint32_t pos = img.u8(t2 + r * width + k);
+  if (pos < F) return img.u32(t2 - 4u - (pos << 2));
+  unsigned long long mine = ~0ull;        // this segment's nearest miss
+  uint32_t mine_p = 0;
+  if (slo == 0u) {                        // the accuracy term vanishes: the fastest entry
+    const uint2 Bv = img.v2(so + SL.bestB);
+    mine = (unsigned long long)Bv.x * 10000ull;
+    mine_p = Bv.y;
+  } else {
     uint32_t acc_floor = 0;               // candidates that miss both need accuracy >= this
     uint32_t pred_cap = 0xFFFFFFFFu;      // ... and latency <= this
     if (r > 0) {                          // some entry meets the SLO (and misses the accuracy)
       const uint32_t A = img.u32(so + SL.bestA + (r << 2));
-      best = (unsigned long long)slo * (min_acc - (A & 0xFFFFu));
-      best_p = A >> 16;
+      mine = (unsigned long long)slo * (min_acc - (A & 0xFFFFu));
+      mine_p = A >> 16;
       acc_floor = (A & 0xFFFFu) + 1u;
     }
     if (k < Ka) {                         // some entry meets the accuracy (and misses the SLO)
       const uint2 Bv = img.v2(so + SL.bestB + (k << 3));
       const unsigned long long d = (unsigned long long)(Bv.x - slo) * 10000ull;
-      if (d < best || (d == best && Bv.y < best_p)) { best = d; best_p = Bv.y; }
+      if (d < mine || (d == mine && Bv.y < mine_p)) { mine = d; mine_p = Bv.y; }
       pred_cap = Bv.x;
     }
-    for (uint32_t o = img.u8(so + SL.ordStart + r); o < sl.w; ++o) {   // stair entries above the SLO, ascending
+    for (uint32_t o = img.u8(so + SL.ordStart + r); o < Fs; ++o) {   // stair entries above the SLO, ascending
       const uint2 e = img.v2(so + SL.walk + (o << 3));
       if (e.x > pred_cap) break;
       const unsigned long long over = (unsigned long long)(e.x - slo) * 10000ull;
-      if (over > best) break;             // later entries overshoot the SLO even more
+      if (over > mine) break;             // later entries overshoot the SLO even more
       const uint32_t acc = e.y & 0xFFFFu, p = e.y >> 16;
       if (acc >= acc_floor && acc < min_acc) {
         const unsigned long long d = over + (unsigned long long)slo * (min_acc - acc);
-        if (d < best || (d == best && p < best_p)) { best = d; best_p = p; }
+        if (d < mine || (d == mine && p < mine_p)) { mine = d; mine_p = p; }
       }
     }
-    return INFAAS_NO_FEASIBLE | img.u32(t2 - 4u - (best_p << 2));
+  }
+  if (mine < best) { best = mine; best_id = img.u32(t2 - 4u - (mine_p << 2)); }
+  return PENDING;
+}
+
+template <class Img>
+__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t task,
+                                                uint32_t slo, uint32_t min_acc) {
+  if (task >= c.n_tasks) return INFAAS_INVALID;
+  uint4 sl = __ldg(c.slow + task);
+  if (sl.z & TASK_FLAG_INVALID) return INFAAS_INVALID;
+  unsigned long long best = ~0ull;
+  uint32_t best_p = 0;
+  if (!(sl.z & TASK_FLAG_NOT_INDEXED)) {
+    // the list's segments in order: the first has its header in the image, the others
+    // (lists longer than INDEX_MAX_F) in global memory
+    uint4 h = img.v4(task * HDR_BYTES + ((threadIdx.x & 7u) << 4));   // this lane's copy
+    for (;;) {
+      const uint32_t d = slow_segment(img, sl, h, slo, min_acc, best, best_p);
+      if (d != PENDING) return d;
+      const uint32_t next = sl.w >> 8;                       // 1 + index of the next segment
+      if (next == 0u) break;
+      sl = __ldg(c.slow + c.n_tasks + next - 1u);
+      h = __ldg(c.xhdr + next - 1u);
+    }
+    return INFAAS_NO_FEASIBLE | best_p;
   }
   const uint32_t F = __ldg(c.f_len + task);
   const uint32_t V = __ldg(c.task_off + task + 1) - __ldg(c.task_off + task);

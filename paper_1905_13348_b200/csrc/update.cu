@@ -215,8 +215,13 @@ __device__ __forceinline__ uint32_t group8_or(uint32_t v) {
 // accuracies span more than the bitmap supports, or the block lies beyond what the 16-bit
 // offsets address.  blockDim = REBUILD_THREADS: the pair loops give every entry 8 lanes, and
 // the tables, which do not depend on each other, are written by different groups of warps.
-__device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, IndexScratch &S) {
+// `xi`: 0xFFFFFFFF for the task's first segment (header and SLO records go into the image), else
+// the index of this further segment (header to xhdr[xi], no records: only the slow path comes
+// here).  `next`: 1 + index of the task's next segment, 0 if this is the last.
+__device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, IndexScratch &S, uint32_t xi,
+                            uint32_t next) {
   const uint32_t tid = threadIdx.x, B = blockDim.x;
+  const bool first = xi == 0xFFFFFFFFu;
   const uint32_t sub = tid & 7u, PB = B >> 3;          // lane of the entry's group; entries per pass
   // distinct values ...
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {            // uniform trip count
@@ -328,7 +333,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
 
   // SLO records (see common.cuh)
   uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
-  share(B / 2, B / 4, SLO_BUCKETS, [&](uint32_t j) {
+  share(B / 2, B / 4, first ? SLO_BUCKETS : 0u, [&](uint32_t j) {
     uint32_t lb = 0, cnt = 0, thr = 0;
     for (uint32_t i = 0; i < Ks; ++i) {
       const uint32_t b = S.bucket[i];
@@ -394,9 +399,12 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   share(15 * B / 16, B / 16, Ks, [&](uint32_t i) { Pd_g[i] = S.Pd[i]; });
 
   const uint32_t cb = ((BL.bitmap - BL.t2) >> 2) + CB_BIAS - acc_lo / ACC_WORD_BITS;
-  write_header(c, t, make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
-                                ((base + BL.t2) >> 4) | (width << 16) | (nbw << 24), acc_lo | (cb << 16)));
-  if (tid == 0) c.slow[t] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs);
+  const uint4 hdr = make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
+                               ((base + BL.t2) >> 4) | (width << 16) | (nbw << 24), acc_lo | (cb << 16));
+  if (first) write_header(c, t, hdr);
+  else if (tid == 0) c.xhdr[xi] = hdr;
+  if (tid == 0)
+    c.slow[first ? t : c.n_tasks + xi] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs | (next << 8));
   return true;
 }
 
@@ -523,7 +531,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   if ((tid & 31) == 0 && my_kept) atomicAdd(&s_total, my_kept);
   __syncthreads();
   const uint32_t F = s_total;
-  bool indexed = F > 0 && F <= INDEX_MAX_F;
+  bool indexed = F > 0;
   unsigned char *region = c.regions + c.reg_off[t];
 
   // 4. compact into the task's region (scan order): keys and ids
@@ -534,7 +542,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     const uint32_t id = c.s_id[base + (v32 & 0xFFFFu)];
     keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
     ids_g[pos] = id;
-    if (indexed) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }
+    if (pos < INDEX_MAX_F) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }   // first segment
   };
   uint32_t kept_so_far = 0;
   for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
@@ -565,7 +573,22 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     if (i < F && sidx == 0) emit(rank, a64, a32);
     __syncthreads();
   }
-  if (indexed) indexed = build_index(c, t, F, S);
+  // index the list segment by segment (INDEX_MAX_F positions each; almost always one)
+  if (indexed) {
+    const uint32_t segs = (F + INDEX_MAX_F - 1u) / INDEX_MAX_F, x0 = c.seg_base[t];
+    for (uint32_t sg = 0; sg < segs && indexed; ++sg) {
+      const uint32_t off = sg * INDEX_MAX_F, Fseg = min(INDEX_MAX_F, F - off);
+      if (sg) {                                   // later segments: back from the task's region
+        __syncthreads();
+        for (uint32_t i = tid; i < Fseg; i += B) {
+          const unsigned long long e = keys_g[off + i];
+          S.ids[i] = ids_g[off + i]; S.pred[i] = (uint32_t)e; S.acc[i] = (uint16_t)(e >> 32);
+        }
+        __syncthreads();
+      }
+      indexed = build_index(c, t, Fseg, S, sg ? x0 + sg - 1u : 0xFFFFFFFFu, sg + 1u < segs ? x0 + sg + 1u : 0u);
+    }
+  }
   if (!indexed) {
     // no index: header and records that make every query of this task read "none"
     write_header(c, t, dummy_header(c.n_tasks));
