@@ -1,2 +1,3 @@
 """CPU oracle (test infrastructure only; never imported by the CUDA path)."""
-from .oracle import OracleCatalog, build, pred_lat  # noqa: F401
+from .oracle import (ACTIVE, INACTIVE, INTERFERED, OVERLOADED, OracleCatalog,  # noqa: F401
+                     StatefulOracleCatalog, build, pred_lat)

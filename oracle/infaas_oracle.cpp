@@ -18,11 +18,14 @@
 //     latency is suggested (Section 4.1, last sentence of the first paragraph).
 //   * Load per variant is tracked from the queries it serves and its batch size, and is
 //     refreshed periodically (Section 4.2.2, scaling-up algorithm; Section 5).
+//   * Variants have a life cycle (Inactive, Active, Overloaded, Interfered); selection looks
+//     at Active variants first, then at Inactive ones with their loading latency added, and
+//     avoids Overloaded and Interfered ones (Section 4, state machine; Section 4.1).
 //
 // Everything is brute force over the full, unsorted, unpruned catalog.  There is no
 // sorting, no pruning, no early exit and no blocking.  Readings of points the paper leaves
-// open (ties, the queueing term, the distance used for "closest", the queue recursion) are
-// this build's choices; those constants are "parity unpinned" by the paper itself, the
+// open (ties, the queueing term, the distance used for "closest", the queue recursion, what
+// moves a variant between states) are this build's choices; those constants are "parity unpinned" by the paper itself, the
 // structure around them is pinned by the tests under tests/ (worked example of Table 2,
 // brute-force enumeration, closed forms, exact-rational ordering).
 //
@@ -113,6 +116,69 @@ uint32_t select_one(const Row *rows, const uint32_t *queued, const std::vector<u
   return have_feasible ? arg_f : (NO_FEASIBLE_BIT | arg_m);
 }
 
+// ---- state-aware selection (Section 4, "State machine for the lifecycle of model-variants";
+// Section 4.1, Case I and "Mitigating performance degradation") ----
+// Every variant is in one of four states.  A query is answered in this order:
+//   1. Active variants carry no loading latency: among those that meet both requirements,
+//      the one with the smallest (cost, pred, 10000-acc, id) -- as in select_one.
+//   2. Otherwise Inactive variants, which must be loaded first: with eff = min(2^32-1,
+//      pred + load_lat), among those with eff <= slo and acc >= min_acc the one with the
+//      lowest combined latency: smallest (eff, 10000-acc, id).
+//   3. Otherwise a suggestion (bit 31 set): over the Active and Inactive variants, the one
+//      with the smallest distance d = 10000*max(0,L-slo) + slo*max(0,min_acc-acc), L = pred
+//      for Active and eff for Inactive; equal distances go to an Active variant before an
+//      Inactive one, then by the order of step 1 / step 2.
+// Overloaded and Interfered variants are never chosen nor suggested.  A task with no Active
+// or Inactive variant answers INVALID.
+const uint8_t ST_INACTIVE = 0, ST_ACTIVE = 1, ST_OVERLOADED = 2, ST_INTERFERED = 3;
+
+struct Key6 {
+  uint64_t k[6];
+};
+bool key6_less(const Key6 &a, const Key6 &b) {
+  for (int i = 0; i < 6; ++i) {
+    if (a.k[i] < b.k[i]) return true;
+    if (a.k[i] > b.k[i]) return false;
+  }
+  return false;
+}
+
+uint32_t select_one_stateful(const Row *rows, const uint32_t *queued, const uint8_t *state,
+                             const uint32_t *load_lat, const std::vector<uint32_t> &members,
+                             uint32_t slo, uint16_t min_acc) {
+  bool have_active = false, have_inactive = false, have_any = false;
+  Key6 best_a{}, best_i{}, best_m{};
+  uint32_t arg_a = 0, arg_i = 0, arg_m = 0;
+  for (uint32_t v : members) {
+    const Row &r = rows[v];
+    if (state[v] != ST_ACTIVE && state[v] != ST_INACTIVE) continue;
+    const bool active = state[v] == ST_ACTIVE;
+    uint32_t p = pred_lat(r.lat_us, queued[v], r.batch);
+    uint64_t e = (uint64_t)p + (uint64_t)load_lat[v];
+    if (e > U32_MAX) e = U32_MAX;
+    uint64_t L = active ? (uint64_t)p : e;               // latency the query would see
+    uint64_t inv_acc = (uint64_t)(10000 - (int)r.acc_bp);
+    bool ok = (L <= slo) && (r.acc_bp >= min_acc);
+    if (ok && active) {
+      Key6 k{{r.cost, p, inv_acc, v, 0, 0}};
+      if (!have_active || key6_less(k, best_a)) { best_a = k; arg_a = v; have_active = true; }
+    }
+    if (ok && !active) {
+      Key6 k{{e, inv_acc, v, 0, 0, 0}};
+      if (!have_inactive || key6_less(k, best_i)) { best_i = k; arg_i = v; have_inactive = true; }
+    }
+    uint64_t over_lat = L > slo ? L - slo : 0;
+    uint64_t under_acc = min_acc > r.acc_bp ? (uint64_t)(min_acc - r.acc_bp) : 0;
+    uint64_t d = 10000ull * over_lat + (uint64_t)slo * under_acc;
+    Key6 k = active ? Key6{{d, 0, r.cost, p, inv_acc, v}} : Key6{{d, 1, e, inv_acc, v, 0}};
+    if (!have_any || key6_less(k, best_m)) { best_m = k; arg_m = v; have_any = true; }
+  }
+  if (have_active) return arg_a;
+  if (have_inactive) return arg_i;
+  if (have_any) return NO_FEASIBLE_BIT | arg_m;
+  return INVALID;
+}
+
 std::vector<std::vector<uint32_t>> members_by_task(const Row *rows, uint32_t n_variants,
                                                    uint32_t n_tasks) {
   std::vector<std::vector<uint32_t>> m(n_tasks);
@@ -187,6 +253,52 @@ void oracle_load_update(const void *rows_v, uint32_t n_variants, uint32_t *queue
     if (arrived > U32_MAX) arrived = U32_MAX;
     queued[v] = (uint32_t)(arrived > drain ? arrived - drain : 0);
     served_total[v] += count[v];
+  }
+}
+
+// State-aware form of oracle_select: `state` and `load_lat_us` hold one entry per variant.
+void oracle_select_stateful(const void *rows_v, uint32_t n_variants, uint32_t n_tasks,
+                            const uint32_t *queued, const uint8_t *state, const uint32_t *load_lat_us,
+                            const uint16_t *task, const uint32_t *slo_us, const uint16_t *min_acc_bp,
+                            uint64_t n, uint32_t *decision, int n_threads) {
+  const Row *rows = (const Row *)rows_v;
+  auto members = members_by_task(rows, n_variants, n_tasks);
+  auto work = [&](uint64_t lo, uint64_t hi) {
+    for (uint64_t q = lo; q < hi; ++q) {
+      if (task[q] >= n_tasks) {
+        decision[q] = INVALID;
+        continue;
+      }
+      decision[q] = select_one_stateful(rows, queued, state, load_lat_us, members[task[q]], slo_us[q],
+                                        min_acc_bp[q]);
+    }
+  };
+  if (n_threads <= 1) {
+    work(0, n);
+    return;
+  }
+  std::vector<std::thread> th;
+  for (int i = 0; i < n_threads; ++i)
+    th.emplace_back(work, n * (uint64_t)i / n_threads, n * (uint64_t)(i + 1) / n_threads);
+  for (auto &t : th) t.join();
+}
+
+// State-aware end of a window: oracle_load_update, then every variant's state follows its
+// load (Section 4: a variant is Active once loaded, Overloaded while it serves at its peak
+// throughput):
+//   Inactive and it was given queries this window          -> Active (it has been loaded)
+//   then, Active or Overloaded: queue not empty afterwards -> Overloaded, else Active
+//   Interfered stays (it is set from outside, by monitoring).
+void oracle_load_update_stateful(const void *rows_v, uint32_t n_variants, uint32_t *queued,
+                                 uint64_t *served_total, uint64_t counters[3], uint8_t *state,
+                                 const uint32_t *decision, uint64_t n, uint32_t window_us) {
+  std::vector<uint64_t> before(served_total, served_total + n_variants);
+  oracle_load_update(rows_v, n_variants, queued, served_total, counters, decision, n, window_us);
+  for (uint32_t v = 0; v < n_variants; ++v) {
+    uint64_t count = served_total[v] - before[v];
+    if (state[v] == ST_INACTIVE && count > 0) state[v] = ST_ACTIVE;
+    if (state[v] == ST_ACTIVE || state[v] == ST_OVERLOADED)
+      state[v] = queued[v] > 0 ? ST_OVERLOADED : ST_ACTIVE;
   }
 }
 

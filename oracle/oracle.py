@@ -21,6 +21,8 @@ _lib = None
 
 NO_FEASIBLE_BIT = 0x80000000
 INVALID = 0xFFFFFFFF
+# life-cycle states of a variant (Section 4, state machine)
+INACTIVE, ACTIVE, OVERLOADED, INTERFERED = 0, 1, 2, 3
 
 
 def build(force: bool = False) -> str:
@@ -48,6 +50,15 @@ def _load():
         lib.oracle_load_update.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
                                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                            ctypes.c_uint64, ctypes.c_uint32]
+        lib.oracle_select_stateful.restype = None
+        lib.oracle_select_stateful.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
+                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                               ctypes.c_uint64, ctypes.c_void_p, ctypes.c_int]
+        lib.oracle_load_update_stateful.restype = None
+        lib.oracle_load_update_stateful.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
+                                                    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                    ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32]
         _lib = lib
     return _lib
 
@@ -95,3 +106,35 @@ class OracleCatalog:
         _load().oracle_load_update(_ptr(self.rows), self.n_variants, _ptr(self.queued),
                                    _ptr(self.served_total), _ptr(self.counters),
                                    _ptr(decision), decision.shape[0], int(window_us))
+
+
+class StatefulOracleCatalog(OracleCatalog):
+    """Catalog with a life-cycle state and a loading latency per variant (Section 4, state
+    machine; Section 4.1, Case I): `select` looks at Active variants, then at Inactive ones,
+    then suggests; `load_update` also moves the states."""
+
+    def __init__(self, rows: np.ndarray, n_tasks: int, state, load_lat_us):
+        super().__init__(rows, n_tasks)
+        self.state = np.ascontiguousarray(state, np.uint8).copy()
+        self.load_lat_us = np.ascontiguousarray(load_lat_us, np.uint32).copy()
+        assert self.state.shape == (self.n_variants,) and self.load_lat_us.shape == (self.n_variants,)
+
+    def select(self, task, slo_us, min_acc_bp, n_threads: int = 1) -> np.ndarray:
+        task = np.ascontiguousarray(task, np.uint16)
+        slo_us = np.ascontiguousarray(slo_us, np.uint32)
+        min_acc_bp = np.ascontiguousarray(min_acc_bp, np.uint16)
+        n = task.shape[0]
+        assert slo_us.shape[0] == n and min_acc_bp.shape[0] == n
+        out = np.empty(n, np.uint32)
+        _load().oracle_select_stateful(_ptr(self.rows), self.n_variants, self.n_tasks,
+                                       _ptr(self.queued), _ptr(self.state), _ptr(self.load_lat_us),
+                                       _ptr(task), _ptr(slo_us), _ptr(min_acc_bp), n, _ptr(out),
+                                       int(n_threads))
+        return out
+
+    def load_update(self, decision, window_us: int) -> None:
+        decision = np.ascontiguousarray(decision, np.uint32)
+        _load().oracle_load_update_stateful(_ptr(self.rows), self.n_variants, _ptr(self.queued),
+                                            _ptr(self.served_total), _ptr(self.counters),
+                                            _ptr(self.state), _ptr(decision), decision.shape[0],
+                                            int(window_us))
