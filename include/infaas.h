@@ -58,6 +58,7 @@ typedef struct {
 #define INFAAS_E_ALIGN (-8)     /* a device array is not 16-byte aligned                  */
 #define INFAAS_E_DEVICE (-9)    /* a kernel reported an internal error (a bounded wait ran
                                    out); the catalog is unchanged by that call            */
+#define INFAAS_E_BAD_STATE (-10) /* a variant state is not one of INFAAS_STATE_*          */
 
 /* Limits. */
 #define INFAAS_MAX_VARIANTS 0x7FFFFFFEu   /* ids must fit below bit 31                     */
@@ -138,6 +139,45 @@ int infaas_tally(infaas_catalog *c, const uint32_t *d_decision, uint64_t n, void
 int infaas_pending_counts(infaas_catalog *c, uint32_t *d_counts, int set, void *cuda_stream);
 int infaas_advance(infaas_catalog *c, uint32_t window_us, void *cuda_stream);
 
+/* Life cycle of a variant (Section 4, "State machine for the lifecycle of model-variants"):
+ * Inactive = not loaded, Active = loaded and below its peak throughput, Overloaded = serving
+ * at its peak throughput, Interfered = slower than profiled because of co-located work. */
+#define INFAAS_STATE_INACTIVE 0
+#define INFAAS_STATE_ACTIVE 1
+#define INFAAS_STATE_OVERLOADED 2
+#define INFAAS_STATE_INTERFERED 3
+
+/* Give every variant a state and a loading latency, and switch the catalog to state-aware
+ * selection (Section 4.1, Case I and "Mitigating performance degradation").  From then on
+ * infaas_select_batch answers a query in this order:
+ *   1. among the Active variants of its task that meet both requirements, the one with the
+ *      smallest (cost, pred_lat, 10000-acc, id) -- Active variants carry no loading latency;
+ *   2. otherwise, among the Inactive variants with  eff = min(2^32-1, pred_lat + load_lat)
+ *      <= slo and acc >= min_acc, the one with the lowest combined loading and inference
+ *      latency: smallest (eff, 10000-acc, id);
+ *   3. otherwise bit 31 set and the nearest miss over the Active and Inactive variants:
+ *      smallest d = 10000*max(0,L-slo) + slo*max(0,min_acc-acc) with L = pred_lat (Active) or
+ *      eff (Inactive); equal d goes to an Active variant first, then by the order of 1. / 2.
+ * Overloaded and Interfered variants are neither chosen nor suggested; a task without an
+ * Active or Inactive variant answers INFAAS_INVALID.  And infaas_load_update / infaas_advance,
+ * after the queue recursion, move the states with the load:
+ *     Inactive and count(v) > 0                      -> Active   (it was loaded to serve them)
+ *     then, Active or Overloaded: queued(v) > 0      -> Overloaded, else Active
+ *     Interfered is left alone (set it from outside with this call).
+ * A catalog on which this was never called behaves as if every variant were Active and
+ * never changes a state.
+ *   h_state        HOST, n_variants bytes indexed by variant id, each an INFAAS_STATE_* value.
+ *   h_load_lat_us  HOST, n_variants u32 indexed by variant id (time to load the variant,
+ *                  microseconds), or NULL for all zero.  Both are copied.
+ * Rebuilds the scan lists; synchronises cuda_stream.  Errors: E_NULL, E_BAD_STATE (nothing is
+ * changed), E_CUDA. */
+int infaas_catalog_set_states(infaas_catalog *c, const uint8_t *h_state,
+                              const uint32_t *h_load_lat_us, void *cuda_stream);
+
+/* Copy the variants' states to HOST: h_state[n_variants] indexed by variant id (all Active
+ * if infaas_catalog_set_states was never called).  Synchronises cuda_stream. */
+int infaas_catalog_get_states(infaas_catalog *c, uint8_t *h_state, void *cuda_stream);
+
 /* Copy the load state to HOST arrays (any of the four may be NULL to skip it):
  *   h_queued[n_variants], h_pred_lat_us[n_variants], h_served_total[n_variants] indexed by
  *   variant id; h_counters[3] = feasible decisions tallied, NO_FEASIBLE decisions seen,
@@ -148,7 +188,8 @@ int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_
                              uint64_t *h_served_total, uint64_t h_counters[3],
                              void *cuda_stream);
 
-/* Copy one task's scan list to HOST: the ids of its non-dominated variants in scan order.
+/* Copy one task's scan list to HOST: the ids of its non-dominated variants in scan order
+ * (state-aware catalogs: the Active list, then the Inactive list).
  * h_ids may be NULL to query the length only; at most `cap` ids are written.
  * *h_len receives the list's length.  Synchronises cuda_stream.  For inspection/tests. */
 int infaas_catalog_get_frontier(infaas_catalog *c, uint32_t task, uint32_t *h_ids,

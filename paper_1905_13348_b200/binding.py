@@ -16,13 +16,15 @@ from .build import LIB_PATH
 
 NO_FEASIBLE = 0x80000000
 INVALID = 0xFFFFFFFF
+STATE_INACTIVE, STATE_ACTIVE, STATE_OVERLOADED, STATE_INTERFERED = 0, 1, 2, 3
 
 _lib = None
 
 EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
            "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info",
-           "infaas_tally", "infaas_pending_counts", "infaas_advance")
+           "infaas_tally", "infaas_pending_counts", "infaas_advance",
+           "infaas_catalog_set_states", "infaas_catalog_get_states")
 
 
 class InfaasError(RuntimeError):
@@ -60,6 +62,9 @@ def _load():
     lib.infaas_advance.argtypes = [vp, u32, vp]
     for name in ("infaas_tally", "infaas_pending_counts", "infaas_advance"):
         getattr(lib, name).restype = i32
+    lib.infaas_catalog_set_states.argtypes = [vp, vp, vp, vp]
+    lib.infaas_catalog_get_states.argtypes = [vp, vp, vp]
+    lib.infaas_catalog_set_states.restype = lib.infaas_catalog_get_states.restype = i32
     lib.infaas_tally_static.argtypes = [vp, u64, u32, vp, vp, i32, vp]
     lib.infaas_tally_static.restype = i32
     lib.infaas_strerror.argtypes = [i32]
@@ -153,6 +158,27 @@ def infaas_pending_counts(cat: Catalog, d_counts, set: bool, stream=None) -> Non
 
 def infaas_advance(cat: Catalog, window_us: int, stream=None) -> None:
     _check(_load().infaas_advance(cat.handle, int(window_us), _stream_ptr(stream)), "infaas_advance")
+
+
+def infaas_catalog_set_states(cat: Catalog, state, load_lat_us=None, stream=None) -> None:
+    """state: host array of n_variants INFAAS_STATE_* bytes; load_lat_us: host u32 array or None."""
+    state = np.ascontiguousarray(state, np.uint8)
+    if state.shape != (cat.n_variants,):
+        raise ValueError("state must have n_variants entries")
+    if load_lat_us is not None:
+        load_lat_us = np.ascontiguousarray(load_lat_us, np.uint32)
+        if load_lat_us.shape != (cat.n_variants,):
+            raise ValueError("load_lat_us must have n_variants entries")
+    _check(_load().infaas_catalog_set_states(cat.handle, state.ctypes.data,
+                                             None if load_lat_us is None else load_lat_us.ctypes.data,
+                                             _stream_ptr(stream)), "infaas_catalog_set_states")
+
+
+def infaas_catalog_get_states(cat: Catalog, stream=None) -> np.ndarray:
+    state = np.empty(cat.n_variants, np.uint8)
+    _check(_load().infaas_catalog_get_states(cat.handle, state.ctypes.data, _stream_ptr(stream)),
+           "infaas_catalog_get_states")
+    return state
 
 
 def infaas_catalog_get_state(cat: Catalog, stream=None) -> dict:

@@ -86,6 +86,7 @@ const char *infaas_strerror(int code) {
     case INFAAS_E_CUDA: return "CUDA call failed (see infaas_last_cuda_error)";
     case INFAAS_E_ALIGN: return "device array is not 16-byte aligned";
     case INFAAS_E_DEVICE: return "a kernel reported an internal error";
+    case INFAAS_E_BAD_STATE: return "variant state is not one of INFAAS_STATE_*";
     default: return "unknown error code";
   }
 }
@@ -149,10 +150,10 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   std::vector<uint32_t> seg_base(n_tasks + 1, 0);
   for (uint32_t t = 0; t < n_tasks; ++t) {
     const uint32_t V = task_off[t + 1] - task_off[t];
-    const uint32_t segs = V ? (V + infaas::INDEX_MAX_F - 1) / infaas::INDEX_MAX_F : 1;
+    // a state-aware catalog has two lists per task (V entries together): one segment more
+    const uint32_t segs = (V + infaas::INDEX_MAX_F - 1) / infaas::INDEX_MAX_F + 1;
     seg_base[t + 1] = seg_base[t] + segs - 1;
-    worst_image += (uint64_t)(segs - 1) * infaas::block_capacity(infaas::INDEX_MAX_F) +
-                   infaas::block_capacity(V - (segs - 1) * infaas::INDEX_MAX_F);
+    worst_image += (uint64_t)segs * infaas::block_capacity(V);
   }
   const uint32_t n_extra = seg_base[n_tasks];
   if (worst_image > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
@@ -164,6 +165,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_id = carve((size_t)n_variants * 4), o_queued = carve((size_t)n_variants * 4);
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
+  const size_t o_state = carve((size_t)n_variants), o_load_lat = carve((size_t)n_variants * 4);
   const size_t o_regions = carve((size_t)region_bytes);
   const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve(((size_t)n_tasks + n_extra) * 16);
   const size_t o_seg_base = carve((n_tasks + 1) * 4), o_xhdr = carve((size_t)n_extra * 16 + 16);
@@ -182,6 +184,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   LOAD_TRY(cudaMalloc(&c->arena, total));
   unsigned char *base = static_cast<unsigned char *>(c->arena);
   LOAD_TRY(cudaMemset(base, 0, total));
+  LOAD_TRY(cudaMemset(base + o_state, INFAAS_STATE_ACTIVE, n_variants));
   LOAD_TRY(cudaMemcpy(base + o_task_off, task_off.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_reg_off, reg_off.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_seg_base, seg_base.data(), (n_tasks + 1) * 4, cudaMemcpyHostToDevice));
@@ -207,6 +210,9 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.s_pred = reinterpret_cast<uint32_t *>(base + o_pred);
   d.s_served = reinterpret_cast<unsigned long long *>(base + o_served);
   d.count_by_id = reinterpret_cast<uint32_t *>(base + o_count);
+  d.stateful = 0;
+  d.s_state = base + o_state;
+  d.s_load_lat = reinterpret_cast<const uint32_t *>(base + o_load_lat);
   d.regions = base + o_regions;
   d.f_len = reinterpret_cast<uint32_t *>(base + o_flen);
   d.slow = reinterpret_cast<uint4 *>(base + o_slow);
@@ -285,6 +291,43 @@ int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n
                        uint32_t window_us, void *cuda_stream) {
   const int rc = infaas_tally(c, d_decision, n, cuda_stream);
   return rc != INFAAS_OK ? rc : infaas_advance(c, window_us, cuda_stream);
+}
+
+int infaas_catalog_set_states(infaas_catalog *c, const uint8_t *h_state, const uint32_t *h_load_lat_us,
+                              void *cuda_stream) {
+  if (!c || !h_state) return INFAAS_E_NULL;
+  const uint32_t nv = c->d.n_variants;
+  for (uint32_t v = 0; v < nv; ++v)
+    if (h_state[v] > INFAAS_STATE_INTERFERED) return INFAAS_E_BAD_STATE;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  std::vector<unsigned char> st(nv);
+  std::vector<uint32_t> ll(nv, 0u);
+  for (uint32_t v = 0; v < nv; ++v) {
+    st[c->slot_of_id[v]] = h_state[v];
+    if (h_load_lat_us) ll[c->slot_of_id[v]] = h_load_lat_us[v];
+  }
+  CUDA_TRY(cudaMemcpyAsync(c->d.s_state, st.data(), nv, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(cudaMemcpyAsync(const_cast<uint32_t *>(c->d.s_load_lat), ll.data(), (size_t)nv * 4,
+                           cudaMemcpyHostToDevice, s));
+  c->d.stateful = 1;
+  CUDA_TRY(infaas::launch_rebuild(c->d, /*advance_queues=*/false, 0, s));
+  CUDA_TRY(cudaStreamSynchronize(s));     // the host copies above go out of scope
+  return refresh_select_plan(c, s);
+}
+
+int infaas_catalog_get_states(infaas_catalog *c, uint8_t *h_state, void *cuda_stream) {
+  if (!c || !h_state) return INFAAS_E_NULL;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const uint32_t nv = c->d.n_variants;
+  std::vector<unsigned char> st(nv);
+  CUDA_TRY(cudaMemcpyAsync(st.data(), c->d.s_state, nv, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  for (uint32_t v = 0; v < nv; ++v) h_state[v] = st[c->slot_of_id[v]];
+  return INFAAS_OK;
 }
 
 int infaas_catalog_get_state(infaas_catalog *c, uint32_t *h_queued, uint32_t *h_pred_lat_us,

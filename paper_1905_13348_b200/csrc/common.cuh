@@ -14,6 +14,12 @@ namespace infaas {
 // Scan list of a task: its non-dominated variants sorted by (cost, pred_lat, 10000-acc, id).
 // Position p in that order is what selection returns the smallest feasible of.
 //
+// A state-aware catalog has two lists per task, one after the other: the Active variants in
+// the order above, then the Inactive ones with pred_lat + loading latency (saturating) in
+// place of both cost and pred_lat; each list is pruned on its own, variants in other states
+// are in neither.  "First feasible position, else the smallest distance at the lowest
+// position" over the two lists in this order is the state-aware answer.
+//
 // A list is cut into segments of at most INDEX_MAX_F consecutive positions (almost always
 // one).  The selection kernel's fast path looks at the first segment only; if that holds
 // nothing feasible the slow path goes through the others in order.  For a segment of F
@@ -62,7 +68,8 @@ namespace infaas {
 //                             is word cb - CB_BIAS + a / 24 counted from t2_off)
 //
 // Per task in global memory (`regions`): keys u64[V] (pred_lat | acc_bp << 32, scan order,
-// F used) and ids u32[V], for lists without an index and for inspection.
+// F used; for Inactive entries the latency includes the loading latency) and ids u32[V], for
+// lists without an index and for inspection.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
@@ -153,6 +160,9 @@ struct DeviceCatalog {
   uint32_t *s_pred;
   unsigned long long *s_served;
   uint32_t *count_by_id;     // [n_variants], zero between windows
+  uint32_t stateful;         // 1: states and loading latencies below take part (else all Active)
+  unsigned char *s_state;    // INFAAS_STATE_* per slot
+  const uint32_t *s_load_lat;  // loading latency per slot, microseconds
 
   unsigned char *regions;    // per task: keys u64[V], ids u32[V] (scan order)
   uint32_t *f_len;           // [n_tasks] list length F

@@ -418,7 +418,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
   unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
-  __shared__ uint32_t s_last, s_total;
+  __shared__ uint32_t s_last, s_total, s_inlist;
   __shared__ IndexScratch S;
 
   const uint32_t t = blockIdx.x, tid = threadIdx.x, B = blockDim.x;
@@ -436,149 +436,196 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);
   uint4 *attr = reinterpret_cast<uint4 *>((reinterpret_cast<uintptr_t>(o32 + sort_n) + 15u) & ~(uintptr_t)15u);
 
-  // 1. queue recursion, predicted latency, sort keys
-  for (uint32_t i = tid; i < P; i += B) {
-    if (i < V) {
-      const uint32_t slot = base + i;
-      const uint32_t lat = c.s_lat[slot];
-      const uint32_t batch = c.s_batch[slot];
-      uint32_t queued = c.s_queued[slot];
-      if (advance) {
-        const uint32_t id = c.s_id[slot];
-        const uint32_t cnt = c.count_by_id[id];
-        c.count_by_id[id] = 0;
-        c.s_served[slot] += cnt;
-        unsigned long long arrived = (unsigned long long)queued + cnt;
-        if (arrived > U32_MAX_) arrived = U32_MAX_;
-        unsigned long long drain = (unsigned long long)window_us * batch / lat;
-        if (drain > U32_MAX_) drain = U32_MAX_;
-        queued = arrived > drain ? (uint32_t)(arrived - drain) : 0u;
-        c.s_queued[slot] = queued;
-      }
-      unsigned long long p = (unsigned long long)lat + (unsigned long long)queued * lat / batch;
-      const uint32_t pred = p > U32_MAX_ ? U32_MAX_ : (uint32_t)p;
-      c.s_pred[slot] = pred;
-      const uint32_t cost = c.s_cost[slot], inv = 10000u - c.s_acc[slot];
-      k64[i] = ((unsigned long long)cost << 32) | pred;
-      k32[i] = (inv << 16) | i;
-      if (small) attr[i] = make_uint4(cost, pred, inv, i);
-    } else {
-      k64[i] = ~0ull;
-      k32[i] = ~0u;
-    }
-  }
-  __syncthreads();
-
-  uint32_t my_kept = 0;
-  if (small) {
-    // 3 (small tasks, before any sort).  q dominates p iff cost_q <= cost_p, pred_q <= pred_p,
-    // acc_q >= acc_p and it differs in some attribute or has the smaller id -- which, given
-    // the three inequalities, is the same as its key (cost, pred, 10000-acc, local index)
-    // being smaller.  G lanes share an entry's comparisons.
-    const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
-    uint32_t dom = 0;
-    if (p < V) {
-      const uint4 a = attr[p];
-      for (uint32_t q = sidx; q < V; q += G) {
-        const uint4 b = attr[q];                       // (cost, pred, 10000 - acc, local index)
-        if (b.x <= a.x && b.y <= a.y && b.z <= a.z)    // rare
-          dom |= (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w) ? 1u : 0u;
-      }
-    }
-    for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
-    if (p < V && sidx == 0) { keep[p] = !dom; my_kept = !dom; }
-  } else {
-    // 2. bitonic sort of P keys, ascending in (cost, pred, 10000-acc, local index)
-    for (uint32_t k = 2; k <= P; k <<= 1) {
-      for (uint32_t j = k >> 1; j > 0; j >>= 1) {
-        for (uint32_t x = tid; x < (P >> 1); x += B) {
-          uint32_t i = ((x & ~(j - 1)) << 1) | (x & (j - 1));   // lower index of the pair
-          uint32_t l = i | j;
-          bool up = (i & k) == 0;
-          unsigned long long a64 = k64[i], b64 = k64[l];
-          uint32_t a32 = k32[i], b32 = k32[l];
-          bool swap = up ? key_less(b64, b32, a64, a32) : key_less(a64, a32, b64, b32);
-          if (swap) {
-            k64[i] = b64; k64[l] = a64;
-            k32[i] = b32; k32[l] = a32;
-          }
-        }
-        __syncthreads();
-      }
-    }
-    // 3. prune.  In sorted order every dominator of p sits before p, and every earlier entry
-    // q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not larger by the
-    // sort, and it differs in some attribute or has the smaller id).
-    for (uint32_t p = tid; p < V; p += B) {
-      const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
-      bool kp = true;
-      for (uint32_t q0 = 0; q0 < p && kp; q0 += 8) {     // groups of 8, exit between groups
-        bool dom = false;
-#pragma unroll
-        for (uint32_t j = 0; j < 8; ++j) {
-          const uint32_t q = min(q0 + j, p - 1);          // clamped repeats are harmless
-          dom |= (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
-        }
-        kp = !dom;
-      }
-      keep[p] = kp;
-      my_kept += kp;
-    }
-  }
-  if (tid == 0) s_total = 0;
-  __syncthreads();
-  my_kept = __reduce_add_sync(0xFFFFFFFFu, my_kept);
-  if ((tid & 31) == 0 && my_kept) atomicAdd(&s_total, my_kept);
-  __syncthreads();
-  const uint32_t F = s_total;
-  bool indexed = F > 0;
+  // A state-aware catalog has two lists per task: Active variants keyed (cost, pred, 10000-acc,
+  // id), then Inactive ones keyed by their combined loading + inference latency, which takes
+  // the place of both cost and pred.  Each goes through steps 1-4 on its own.
   unsigned char *region = c.regions + c.reg_off[t];
-
-  // 4. compact into the task's region (scan order): keys and ids
   unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(region);
   uint32_t *ids_g = reinterpret_cast<uint32_t *>(region + 8u * V);
-  auto emit = [&](uint32_t pos, unsigned long long v64, uint32_t v32) {   // list position pos
-    const uint32_t pred_p = (uint32_t)v64, acc = 10000u - (v32 >> 16);
-    const uint32_t id = c.s_id[base + (v32 & 0xFFFFu)];
-    keys_g[pos] = ((unsigned long long)acc << 32) | pred_p;
-    ids_g[pos] = id;
-    if (pos < INDEX_MAX_F) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }   // first segment
-  };
-  uint32_t kept_so_far = 0;
-  for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
-    const uint32_t p = p0 + tid;
-    const bool kp = p < V && keep[p];
-    uint32_t total;
-    const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
-    if (kp) {
-      if (small) { o64[pos] = k64[p]; o32[pos] = k32[p]; }      // survivors, not yet in order
-      else emit(pos, k64[p], k32[p]);
-    }
-    kept_so_far += total;
-  }
-  __syncthreads();
-  if (small) {
-    // 2 (small tasks): the survivors' list positions by counting smaller keys
-    uint32_t PF = 1;
-    while (PF < F) PF <<= 1;
-    const uint32_t G = min(32u, B / PF), i = tid / G, sidx = tid % G;
-    uint32_t rank = 0;
-    unsigned long long a64 = 0;
-    uint32_t a32 = 0;
-    if (i < F) {
-      a64 = o64[i]; a32 = o32[i];
-      for (uint32_t j = sidx; j < F; j += G) rank += key_less(o64[j], o32[j], a64, a32);
-    }
-    for (uint32_t o = G >> 1; o; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
-    if (i < F && sidx == 0) emit(rank, a64, a32);
+  uint32_t F = 0, F0 = 0;                 // entries emitted so far; length of the first list
+  const uint32_t n_lists = c.stateful ? 2u : 1u;
+  for (uint32_t list = 0; list < n_lists; ++list) {
     __syncthreads();
+    if (tid == 0) { s_total = 0; s_inlist = 0; }
+    __syncthreads();
+    // 1. queue recursion and states (first pass), predicted latency, sort keys
+    uint32_t mine = 0;
+    for (uint32_t i = tid; i < P; i += B) {
+      bool in = false;
+      uint32_t cost = 0, lat_key = 0, inv = 0;
+      if (i < V) {
+        const uint32_t slot = base + i;
+        uint32_t pred;
+        if (list == 0) {
+          const uint32_t lat = c.s_lat[slot];
+          const uint32_t batch = c.s_batch[slot];
+          uint32_t queued = c.s_queued[slot];
+          if (advance) {
+            const uint32_t id = c.s_id[slot];
+            const uint32_t cnt = c.count_by_id[id];
+            c.count_by_id[id] = 0;
+            c.s_served[slot] += cnt;
+            unsigned long long arrived = (unsigned long long)queued + cnt;
+            if (arrived > U32_MAX_) arrived = U32_MAX_;
+            unsigned long long drain = (unsigned long long)window_us * batch / lat;
+            if (drain > U32_MAX_) drain = U32_MAX_;
+            queued = arrived > drain ? (uint32_t)(arrived - drain) : 0u;
+            c.s_queued[slot] = queued;
+            if (c.stateful) {
+              // loaded by its first queries; at peak throughput while a backlog remains
+              uint32_t st = c.s_state[slot];
+              if (st == INFAAS_STATE_INACTIVE && cnt > 0) st = INFAAS_STATE_ACTIVE;
+              if (st == INFAAS_STATE_ACTIVE || st == INFAAS_STATE_OVERLOADED)
+                st = queued > 0 ? INFAAS_STATE_OVERLOADED : INFAAS_STATE_ACTIVE;
+              c.s_state[slot] = (unsigned char)st;
+            }
+          }
+          unsigned long long p = (unsigned long long)lat + (unsigned long long)queued * lat / batch;
+          pred = p > U32_MAX_ ? U32_MAX_ : (uint32_t)p;
+          c.s_pred[slot] = pred;
+        } else {
+          pred = c.s_pred[slot];
+        }
+        in = true;
+        cost = c.s_cost[slot]; lat_key = pred; inv = 10000u - c.s_acc[slot];
+        if (c.stateful) {
+          in = c.s_state[slot] == (list == 0 ? INFAAS_STATE_ACTIVE : INFAAS_STATE_INACTIVE);
+          if (list == 1) {
+            const unsigned long long e = (unsigned long long)pred + c.s_load_lat[slot];
+            cost = lat_key = e > U32_MAX_ ? U32_MAX_ : (uint32_t)e;
+          }
+        }
+      }
+      if (in) {
+        k64[i] = ((unsigned long long)cost << 32) | lat_key;
+        k32[i] = (inv << 16) | i;
+        if (small) attr[i] = make_uint4(cost, lat_key, inv, i);
+        ++mine;
+      } else {
+        k64[i] = ~0ull;
+        k32[i] = ~0u;
+        if (small && i < V) attr[i] = make_uint4(~0u, ~0u, ~0u, i);   // in neither comparison
+      }
+    }
+    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if ((tid & 31) == 0 && mine) atomicAdd(&s_inlist, mine);
+    __syncthreads();
+    const uint32_t Vl = s_inlist;           // variants in this list before the prune
+
+    uint32_t my_kept = 0;
+    if (small) {
+      // 3 (small tasks, before any sort).  q dominates p iff cost_q <= cost_p, pred_q <= pred_p,
+      // acc_q >= acc_p and it differs in some attribute or has the smaller id -- which, given
+      // the three inequalities, is the same as its key (cost, pred, 10000-acc, local index)
+      // being smaller.  G lanes share an entry's comparisons.
+      const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
+      uint32_t dom = 0;
+      if (p < V) {
+        const uint4 a = attr[p];
+        if (a.z == ~0u) dom = 1;                         // not in this list
+        else
+          for (uint32_t q = sidx; q < V; q += G) {
+            const uint4 b = attr[q];                       // (cost, pred, 10000 - acc, local index)
+            if (b.x <= a.x && b.y <= a.y && b.z <= a.z)    // rare
+              dom |= (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w) ? 1u : 0u;
+          }
+      }
+      for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
+      if (p < V && sidx == 0) { keep[p] = !dom; my_kept = !dom; }
+    } else {
+      // 2. bitonic sort of P keys, ascending in (cost, pred, 10000-acc, local index); what is
+      // not in this list sorts behind it
+      for (uint32_t k = 2; k <= P; k <<= 1) {
+        for (uint32_t j = k >> 1; j > 0; j >>= 1) {
+          for (uint32_t x = tid; x < (P >> 1); x += B) {
+            uint32_t i = ((x & ~(j - 1)) << 1) | (x & (j - 1));   // lower index of the pair
+            uint32_t l = i | j;
+            bool up = (i & k) == 0;
+            unsigned long long a64 = k64[i], b64 = k64[l];
+            uint32_t a32 = k32[i], b32 = k32[l];
+            bool swap = up ? key_less(b64, b32, a64, a32) : key_less(a64, a32, b64, b32);
+            if (swap) {
+              k64[i] = b64; k64[l] = a64;
+              k32[i] = b32; k32[l] = a32;
+            }
+          }
+          __syncthreads();
+        }
+      }
+      // 3. prune.  In sorted order every dominator of p sits before p, and every earlier entry
+      // q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not larger by the
+      // sort, and it differs in some attribute or has the smaller id).
+      for (uint32_t p = tid; p < V; p += B) {
+        const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
+        bool kp = p < Vl;
+        for (uint32_t q0 = 0; q0 < p && kp; q0 += 8) {     // groups of 8, exit between groups
+          bool dom = false;
+#pragma unroll
+          for (uint32_t j = 0; j < 8; ++j) {
+            const uint32_t q = min(q0 + j, p - 1);          // clamped repeats are harmless
+            dom |= (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
+          }
+          kp = !dom;
+        }
+        keep[p] = kp;
+        my_kept += kp;
+      }
+    }
+    __syncthreads();
+    my_kept = __reduce_add_sync(0xFFFFFFFFu, my_kept);
+    if ((tid & 31) == 0 && my_kept) atomicAdd(&s_total, my_kept);
+    __syncthreads();
+    const uint32_t Fl = s_total;
+
+    // 4. compact into the task's region (scan order, behind the earlier list): keys and ids
+    auto emit = [&](uint32_t pos, unsigned long long v64, uint32_t v32) {   // position pos of this list
+      const uint32_t pred_p = (uint32_t)v64, acc = 10000u - (v32 >> 16);
+      const uint32_t id = c.s_id[base + (v32 & 0xFFFFu)];
+      keys_g[F + pos] = ((unsigned long long)acc << 32) | pred_p;
+      ids_g[F + pos] = id;
+      if (list == 0 && pos < INDEX_MAX_F) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }   // first segment
+    };
+    uint32_t kept_so_far = 0;
+    for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
+      const uint32_t p = p0 + tid;
+      const bool kp = p < V && keep[p];
+      uint32_t total;
+      const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
+      if (kp) {
+        if (small) { o64[pos] = k64[p]; o32[pos] = k32[p]; }      // survivors, not yet in order
+        else emit(pos, k64[p], k32[p]);
+      }
+      kept_so_far += total;
+    }
+    __syncthreads();
+    if (small) {
+      // 2 (small tasks): the survivors' list positions by counting smaller keys
+      uint32_t PF = 1;
+      while (PF < Fl) PF <<= 1;
+      const uint32_t G = min(32u, B / PF), i = tid / G, sidx = tid % G;
+      uint32_t rank = 0;
+      unsigned long long a64 = 0;
+      uint32_t a32 = 0;
+      if (i < Fl) {
+        a64 = o64[i]; a32 = o32[i];
+        for (uint32_t j = sidx; j < Fl; j += G) rank += key_less(o64[j], o32[j], a64, a32);
+      }
+      for (uint32_t o = G >> 1; o; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+      if (i < Fl && sidx == 0) emit(rank, a64, a32);
+      __syncthreads();
+    }
+    if (list == 0) F0 = Fl;
+    F += Fl;
   }
-  // index the list segment by segment (INDEX_MAX_F positions each; almost always one)
+  bool indexed = F > 0;
+  // index the lists segment by segment (INDEX_MAX_F positions each; almost always one)
   if (indexed) {
-    const uint32_t segs = (F + INDEX_MAX_F - 1u) / INDEX_MAX_F, x0 = c.seg_base[t];
-    for (uint32_t sg = 0; sg < segs && indexed; ++sg) {
-      const uint32_t off = sg * INDEX_MAX_F, Fseg = min(INDEX_MAX_F, F - off);
-      if (sg) {                                   // later segments: back from the task's region
+    const uint32_t segs0 = (F0 + INDEX_MAX_F - 1u) / INDEX_MAX_F;
+    const uint32_t nseg = segs0 + (F - F0 + INDEX_MAX_F - 1u) / INDEX_MAX_F, x0 = c.seg_base[t];
+    for (uint32_t sg = 0; sg < nseg && indexed; ++sg) {
+      const uint32_t off = sg < segs0 ? sg * INDEX_MAX_F : F0 + (sg - segs0) * INDEX_MAX_F;
+      const uint32_t Fseg = min(INDEX_MAX_F, (sg < segs0 ? F0 : F) - off);
+      if (sg || F0 == 0) {                        // all but the first list's head: back from the task's region
         __syncthreads();
         for (uint32_t i = tid; i < Fseg; i += B) {
           const unsigned long long e = keys_g[off + i];
@@ -586,7 +633,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
         }
         __syncthreads();
       }
-      indexed = build_index(c, t, Fseg, S, sg ? x0 + sg - 1u : 0xFFFFFFFFu, sg + 1u < segs ? x0 + sg + 1u : 0u);
+      indexed = build_index(c, t, Fseg, S, sg ? x0 + sg - 1u : 0xFFFFFFFFu, sg + 1u < nseg ? x0 + sg + 1u : 0u);
     }
   }
   if (!indexed) {
