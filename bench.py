@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, from the ncu capture summarised in profiles/select_kernel_C3.md, per query (part of
 # the decisions is still in L2 when the kernel ends, hence below 12 B).  Set to None when the
 # kernel changes until the counters are taken again.
-NCU_TRAFFIC_BYTES_PER_QUERY = (134.56e6 + 27.51e6) / (1 << 24)
+NCU_TRAFFIC_BYTES_PER_QUERY = (134.56e6 + 27.22e6) / (1 << 24)
 
 
 def parse_args():
@@ -317,6 +317,7 @@ def run_ours(args):
         out["e2e"] = e2e_leg(P, cat, w, dev, update, max(3, min(10, args.steps)), world, dist)
         if w.window and world == 1:
             out["windowed"] = windowed_leg(P, cat, w, inputs[0], d_dec, world)
+            out["stateful"] = stateful_leg(P, w, inputs, d_dec, local, peak)
     else:
         out["e2e"] = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -423,6 +424,44 @@ def windowed_leg(P, cat, w, inp, d_dec, world):
     return {"value": world * nwin * W_ / (ms * 1e-3), "unit": UNIT, "windows": nwin,
             "window_queries": W_, "us_per_window": 1e3 * ms / nwin, "gpu_launches_per_window": 3,
             "how": "CUDA graph of all windows", "us_per_window_python_calls": 1e3 * eager_ms / nwin}
+
+
+def stateful_leg(P, w, inputs, d_dec, local, peak):
+    """The same workload with a life-cycle state and a loading latency per variant
+    (state-aware selection; states move with the load at every update): the selection kernel
+    over all queries against the initial states, then the stream of windows."""
+    import torch
+    from paper_1905_13348_b200 import workloads as W
+    state, load = W.variant_states(w.n_variants)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks, local)
+    P.infaas_catalog_set_states(cat, state, load)
+    stream = torch.cuda.current_stream()
+    reps = 20
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for k in range(3 + reps):
+        t, s, a = inputs[k & 1]
+        if k >= 3:
+            evs[k - 3][0].record(stream)
+        P.infaas_select_batch(cat, t, s, a, d_dec, stream=stream)
+        if k >= 3:
+            evs[k - 3][1].record(stream)
+    torch.cuda.synchronize()
+    sel_ms = sum(e0.elapsed_time(e1) for e0, e1 in evs) / reps
+    dec = d_dec.cpu().numpy().view(np.uint32)
+    ok = dec[(dec >> 31) == 0]
+    info = P.infaas_catalog_get_info(cat)
+    win = windowed_leg(P, cat, w, inputs[0], d_dec, 1)
+    end = P.infaas_catalog_get_states(cat)
+    cat.free()
+    gbs = ALGO_BYTES_PER_QUERY * w.n_queries / (sel_ms * 1e-3) / 1e9
+    return {"select_ms": sel_ms, "select_gbs": gbs, "select_frac_of_hbm_peak": gbs / peak,
+            "decisions": {"active": int((state[ok] == 1).sum()), "inactive": int((state[ok] == 0).sum()),
+                          "no_feasible": int((((dec >> 31) == 1) & (dec != 0xFFFFFFFF)).sum()),
+                          "invalid": int((dec == 0xFFFFFFFF).sum())},
+            "states_start": np.bincount(state, minlength=4).tolist(),
+            "states_after_windows": np.bincount(end, minlength=4).tolist(),
+            "list_entries": info["list_entries"], "image_bytes": info["image_bytes"],
+            "windowed_us_per_window": win["us_per_window"], "windowed_value": win["value"], "unit": UNIT}
 
 
 def main():

@@ -307,6 +307,21 @@ def config_c5(n_windows: int = 1000, window: int = 65536) -> Workload:
                     "switching between two Zipf(1.5) permutations every 50 windows")
 
 
+# Share of the variants that start Inactive / Active / Overloaded / Interfered in the
+# state-aware runs (codes 0..3 as in include/infaas.h).  The paper prints no such mix; it
+# says that every variant starts Inactive and is loaded on demand, so most are Inactive.
+STATE_MIX = (0.85, 0.05, 0.05, 0.05)
+
+
+def variant_states(n_variants: int, seed: int = 6, mix=STATE_MIX):
+    """A life-cycle state per variant drawn from `mix`, and a loading latency per variant,
+    log-uniform over the range the paper prints for its models (Section 2.1: 590 ms - 11 s)."""
+    rng = _rng(seed)
+    state = np.searchsorted(np.cumsum(mix), rng.random(n_variants), side="right").clip(0, 3).astype(np.uint8)
+    load_lat_us = _log_uniform_int(rng, 590_000, 11_000_000, n_variants)
+    return state, load_lat_us
+
+
 CONFIGS = {"C1": config_c1, "C2": config_c2, "C3": config_c3, "C4": config_c4, "C5": config_c5}
 
 
