@@ -1,3 +1,3 @@
 """CPU oracle (test infrastructure only; never imported by the CUDA path)."""
-from .oracle import (ACTIVE, INACTIVE, INTERFERED, OVERLOADED, OracleCatalog,  # noqa: F401
-                     StatefulOracleCatalog, build, pred_lat)
+from .oracle import (ACTIVE, AUTOSCALE_ESCALATE, AUTOSCALE_NONE, INACTIVE, INTERFERED,  # noqa: F401
+                     OVERLOADED, OracleCatalog, StatefulOracleCatalog, autoscale_step, build, pred_lat)

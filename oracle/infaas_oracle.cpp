@@ -22,6 +22,11 @@
 //     at Active variants first, then at Inactive ones with their loading latency added, and
 //     avoids Overloaded and Interfered ones (Section 4, state machine; Section 4.1).
 //
+//   * Each window the Model-Autoscaler compares the running variants' saturation throughput
+//     with the load they serve and, when the headroom is too small, picks the cheaper of
+//     replicating the running variant and upgrading to a faster one of the same architecture
+//     (Section 4.2.1 cost function and constraints; Section 4.2.2 scaling-up algorithm).
+//
 // Everything is brute force over the full, unsorted, unpruned catalog.  There is no
 // sorting, no pruning, no early exit and no blocking.  Readings of points the paper leaves
 // open (ties, the queueing term, the distance used for "closest", the queue recursion, what
@@ -299,6 +304,78 @@ void oracle_load_update_stateful(const void *rows_v, uint32_t n_variants, uint32
     if (state[v] == ST_INACTIVE && count > 0) state[v] = ST_ACTIVE;
     if (state[v] == ST_ACTIVE || state[v] == ST_OVERLOADED)
       state[v] = queued[v] > 0 ? ST_OVERLOADED : ST_ACTIVE;
+  }
+}
+
+// ---- Model-Autoscaler, scaling-up step (Section 4.2.2, "A Greedy Heuristic", scaling up
+// algorithm; cost function and constraints (1), (2), (4) of Section 4.2.1) ----
+// Per task (application), from the window's per-variant tallies `count`:
+//   Q(v)   = floor(10^9 * batch / lat_us)             saturation throughput, milli-queries/s
+//   L      = floor(10^9 * min(2^32-1, sum count) / window_us)   load served, milli-queries/s
+//   cap    = sum over running variants (instances > 0) of instances * Q   (saturating, 64 bit)
+//   need   = ceil(L * slack_pct / 100)                 (saturating)
+//   cap >= need: headroom suffices, no action (variant = 0xFFFFFFFF, delta = 0).
+// Otherwise deficit = need - cap, and with r = the running variant that served most queries
+// this window (ties: lower id; none if nothing runs), the candidate actions are
+//   replicate r:   delta = ceil(deficit / Q(r))
+//   upgrade to v:  v != r, same architecture as r and Q(v) > Q(r) (any v with Q(v) > 0 if
+//                  nothing runs); delta = ceil(deficit / Q(v)) instances of v are added
+// each only if the variant's profiled latency meets the task's SLO (constraint (2)) and delta
+// fits 32 bits.  The action with the smallest  cost * delta * (10^9 + lambda_milli * load_lat_us)
+// wins -- the paper's C (delta + lambda T_load delta) in units of 10^-9 -- replication first on
+// equal cost, then the lower id.  No candidate: variant = 0xFFFFFFFE (the step to the
+// VM-level autoscaler), delta = 0.
+const uint32_t AUTOSCALE_NONE = 0xFFFFFFFFu, AUTOSCALE_ESCALATE = 0xFFFFFFFEu;
+typedef unsigned __int128 u128;
+const uint64_t U64_MAX = ~0ull;
+
+void oracle_autoscale_step(const void *rows_v, uint32_t n_variants, uint32_t n_tasks,
+                           const uint32_t *count, const uint32_t *instances,
+                           const uint32_t *load_lat_us, const uint32_t *task_slo_us,
+                           uint32_t window_us, uint32_t slack_pct, uint32_t lambda_milli,
+                           uint32_t *action_variant, uint32_t *action_delta) {
+  const Row *rows = (const Row *)rows_v;
+  auto members = members_by_task(rows, n_variants, n_tasks);
+  auto Q = [&](uint32_t v) { return (uint64_t)(1000000000ull * rows[v].batch / rows[v].lat_us); };
+  for (uint32_t t = 0; t < n_tasks; ++t) {
+    action_variant[t] = AUTOSCALE_NONE;
+    action_delta[t] = 0;
+    u128 served = 0, cap = 0;
+    bool have_r = false;
+    uint32_t r = 0;
+    for (uint32_t v : members[t]) {
+      served += count[v];
+      if (instances[v] == 0) continue;
+      cap += (u128)instances[v] * Q(v);
+      if (!have_r || count[v] > count[r]) { r = v; have_r = true; }   // ascending id: ties keep the lower
+    }
+    if (served > U32_MAX) served = U32_MAX;
+    if (cap > U64_MAX) cap = U64_MAX;
+    uint64_t L = (uint64_t)(served * 1000000000ull / window_us);
+    u128 need = ((u128)L * slack_pct + 99) / 100;
+    if (need > U64_MAX) need = U64_MAX;
+    if (cap >= need) continue;
+    u128 deficit = need - cap;
+    bool have_best = false;
+    u128 best_cost = 0;
+    uint32_t best_kind = 0, best_v = 0, best_delta = 0;
+    for (uint32_t v : members[t]) {
+      uint32_t kind;                                        // 0 replicate, 1 upgrade
+      if (have_r && v == r) kind = 0;
+      else if (have_r) {
+        if (rows[v].arch != rows[r].arch || Q(v) <= Q(r)) continue;
+        kind = 1;
+      } else kind = 1;
+      if (Q(v) == 0 || rows[v].lat_us > task_slo_us[t]) continue;
+      u128 delta = (deficit + Q(v) - 1) / Q(v);
+      if (delta > U32_MAX) continue;
+      u128 cost = (u128)rows[v].cost * delta * (1000000000ull + (uint64_t)lambda_milli * load_lat_us[v]);
+      if (!have_best || cost < best_cost || (cost == best_cost && kind < best_kind)) {
+        have_best = true; best_cost = cost; best_kind = kind; best_v = v; best_delta = (uint32_t)delta;
+      }
+    }
+    action_variant[t] = have_best ? best_v : AUTOSCALE_ESCALATE;
+    action_delta[t] = have_best ? best_delta : 0;
   }
 }
 

@@ -23,6 +23,8 @@ NO_FEASIBLE_BIT = 0x80000000
 INVALID = 0xFFFFFFFF
 # life-cycle states of a variant (Section 4, state machine)
 INACTIVE, ACTIVE, OVERLOADED, INTERFERED = 0, 1, 2, 3
+# Model-Autoscaler answers that are not a variant id (Section 4.2.2)
+AUTOSCALE_NONE, AUTOSCALE_ESCALATE = 0xFFFFFFFF, 0xFFFFFFFE
 
 
 def build(force: bool = False) -> str:
@@ -59,6 +61,9 @@ def _load():
         lib.oracle_load_update_stateful.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
                                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                                     ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32]
+        lib.oracle_autoscale_step.restype = None
+        lib.oracle_autoscale_step.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32] + \
+            [ctypes.c_void_p] * 4 + [ctypes.c_uint32] * 3 + [ctypes.c_void_p] * 2
         _lib = lib
     return _lib
 
@@ -138,3 +143,20 @@ class StatefulOracleCatalog(OracleCatalog):
                                             _ptr(self.served_total), _ptr(self.counters),
                                             _ptr(self.state), _ptr(decision), decision.shape[0],
                                             int(window_us))
+
+
+def autoscale_step(rows: np.ndarray, n_tasks: int, count, instances, load_lat_us, task_slo_us,
+                   window_us: int, slack_pct: int = 105, lambda_milli: int = 0):
+    """Scaling-up step of the Model-Autoscaler for every task (Section 4.2.2): returns
+    (variant, delta) arrays of n_tasks; see oracle_autoscale_step in infaas_oracle.cpp."""
+    rows = np.ascontiguousarray(rows)
+    nv = rows.shape[0]
+    count, instances, load_lat_us = (np.ascontiguousarray(a, np.uint32) for a in (count, instances, load_lat_us))
+    task_slo_us = np.ascontiguousarray(task_slo_us, np.uint32)
+    assert count.shape == instances.shape == load_lat_us.shape == (nv,) and task_slo_us.shape == (n_tasks,)
+    assert window_us >= 1
+    variant, delta = np.empty(n_tasks, np.uint32), np.empty(n_tasks, np.uint32)
+    _load().oracle_autoscale_step(_ptr(rows), nv, n_tasks, _ptr(count), _ptr(instances), _ptr(load_lat_us),
+                                  _ptr(task_slo_us), int(window_us), int(slack_pct), int(lambda_milli),
+                                  _ptr(variant), _ptr(delta))
+    return variant, delta
