@@ -59,6 +59,7 @@ typedef struct {
 #define INFAAS_E_DEVICE (-9)    /* a kernel reported an internal error (a bounded wait ran
                                    out); the catalog is unchanged by that call            */
 #define INFAAS_E_BAD_STATE (-10) /* a variant state is not one of INFAAS_STATE_*          */
+#define INFAAS_E_BAD_ARG (-11)   /* a scalar argument is out of range (see the function)  */
 
 /* Limits. */
 #define INFAAS_MAX_VARIANTS 0x7FFFFFFEu   /* ids must fit below bit 31                     */
@@ -177,6 +178,43 @@ int infaas_catalog_set_states(infaas_catalog *c, const uint8_t *h_state,
 /* Copy the variants' states to HOST: h_state[n_variants] indexed by variant id (all Active
  * if infaas_catalog_set_states was never called).  Synchronises cuda_stream. */
 int infaas_catalog_get_states(infaas_catalog *c, uint8_t *h_state, void *cuda_stream);
+
+/* Model-Autoscaler, scaling-up step (Section 4.2.2, "A Greedy Heuristic"; cost function and
+ * constraints (1), (2), (4) of Section 4.2.1).  For every task it compares the saturation
+ * throughput of the running variants with the load the window's tallies show and, when the
+ * headroom is below the slack threshold, picks the cheaper of replicating the running variant
+ * and adding a faster variant of the same architecture:
+ *     Q(v)  = floor(10^9 * batch / lat_us)                   milli-queries/s, profiled
+ *     L     = floor(10^9 * min(2^32-1, sum_v count(v)) / window_us)
+ *     cap   = sum over variants with instances > 0 of instances * Q      (saturating, 64 bit)
+ *     need  = ceil(L * slack_pct / 100)                      (saturating)
+ *   cap >= need: no action, variant = INFAAS_AUTOSCALE_NONE, delta = 0.  Otherwise, with
+ *   deficit = need - cap and r = the running variant with the largest count (ties: lower id;
+ *   none if nothing runs), the candidates are r itself (replicate) and every v != r of r's
+ *   architecture with Q(v) > Q(r) (upgrade; if nothing runs: every v), each only if
+ *   lat_us(v) <= the task's SLO and Q(v) > 0, with delta = ceil(deficit / Q(v)) <= 2^32-1
+ *   instances added.  The smallest  cost * delta * (10^9 + lambda_milli * load_lat_us)  wins
+ *   (the paper's C (delta + lambda T_load delta) in units of 10^-9), replication first on
+ *   equal cost, then the lower id.  No candidate: variant = INFAAS_AUTOSCALE_ESCALATE (the
+ *   case the paper hands to the VM-level autoscaler), delta = 0.
+ * count(v) are the pending tallies: call this after infaas_tally and before infaas_advance
+ * (infaas_load_update does both at once and leaves nothing pending).  The loading latencies are
+ * those of infaas_catalog_set_states (zero if never set).  The actions are only reported; apply
+ * them with infaas_autoscale_config.
+ *   infaas_autoscale_config: h_instances HOST n_variants u32 by variant id (running instances
+ *     N of each variant), h_task_slo_us HOST n_tasks u32 (each application's SLO); copied;
+ *     synchronises cuda_stream.  Errors: E_NULL, E_CUDA.
+ *   infaas_autoscale_step: window_us >= 1 (else E_BAD_ARG); slack_pct = the slack threshold in
+ *     percent (the paper uses 1.05 = 105); lambda_milli = the weight lambda in 1/1000 per second;
+ *     d_variant, d_delta DEVICE, n_tasks u32 each, overwritten.  Asynchronous, stream-ordered,
+ *     allocates nothing.  Errors: E_NULL, E_BAD_ARG (also: config never called), E_CUDA. */
+#define INFAAS_AUTOSCALE_NONE 0xFFFFFFFFu
+#define INFAAS_AUTOSCALE_ESCALATE 0xFFFFFFFEu
+int infaas_autoscale_config(infaas_catalog *c, const uint32_t *h_instances,
+                            const uint32_t *h_task_slo_us, void *cuda_stream);
+int infaas_autoscale_step(infaas_catalog *c, uint32_t window_us, uint32_t slack_pct,
+                          uint32_t lambda_milli, uint32_t *d_variant, uint32_t *d_delta,
+                          void *cuda_stream);
 
 /* Copy the load state to HOST arrays (any of the four may be NULL to skip it):
  *   h_queued[n_variants], h_pred_lat_us[n_variants], h_served_total[n_variants] indexed by

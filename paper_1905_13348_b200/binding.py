@@ -17,6 +17,7 @@ from .build import LIB_PATH
 NO_FEASIBLE = 0x80000000
 INVALID = 0xFFFFFFFF
 STATE_INACTIVE, STATE_ACTIVE, STATE_OVERLOADED, STATE_INTERFERED = 0, 1, 2, 3
+AUTOSCALE_NONE, AUTOSCALE_ESCALATE = 0xFFFFFFFF, 0xFFFFFFFE
 
 _lib = None
 
@@ -24,7 +25,8 @@ EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
            "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info",
            "infaas_tally", "infaas_pending_counts", "infaas_advance",
-           "infaas_catalog_set_states", "infaas_catalog_get_states")
+           "infaas_catalog_set_states", "infaas_catalog_get_states",
+           "infaas_autoscale_config", "infaas_autoscale_step")
 
 
 class InfaasError(RuntimeError):
@@ -65,6 +67,9 @@ def _load():
     lib.infaas_catalog_set_states.argtypes = [vp, vp, vp, vp]
     lib.infaas_catalog_get_states.argtypes = [vp, vp, vp]
     lib.infaas_catalog_set_states.restype = lib.infaas_catalog_get_states.restype = i32
+    lib.infaas_autoscale_config.argtypes = [vp, vp, vp, vp]
+    lib.infaas_autoscale_step.argtypes = [vp, u32, u32, u32, vp, vp, vp]
+    lib.infaas_autoscale_config.restype = lib.infaas_autoscale_step.restype = i32
     lib.infaas_tally_static.argtypes = [vp, u64, u32, vp, vp, i32, vp]
     lib.infaas_tally_static.restype = i32
     lib.infaas_strerror.argtypes = [i32]
@@ -179,6 +184,26 @@ def infaas_catalog_get_states(cat: Catalog, stream=None) -> np.ndarray:
     _check(_load().infaas_catalog_get_states(cat.handle, state.ctypes.data, _stream_ptr(stream)),
            "infaas_catalog_get_states")
     return state
+
+
+def infaas_autoscale_config(cat: Catalog, instances, task_slo_us, stream=None) -> None:
+    """instances: host u32 array of n_variants; task_slo_us: host u32 array of n_tasks."""
+    instances = np.ascontiguousarray(instances, np.uint32)
+    task_slo_us = np.ascontiguousarray(task_slo_us, np.uint32)
+    if instances.shape != (cat.n_variants,) or task_slo_us.shape != (cat.n_tasks,):
+        raise ValueError("instances needs n_variants entries and task_slo_us n_tasks")
+    _check(_load().infaas_autoscale_config(cat.handle, instances.ctypes.data, task_slo_us.ctypes.data,
+                                           _stream_ptr(stream)), "infaas_autoscale_config")
+
+
+def infaas_autoscale_step(cat: Catalog, window_us: int, slack_pct: int, lambda_milli: int, d_variant, d_delta,
+                          stream=None) -> None:
+    """d_variant, d_delta: int32/uint32 CUDA tensors of n_tasks, overwritten."""
+    if d_variant.numel() < cat.n_tasks or d_delta.numel() < cat.n_tasks:
+        raise ValueError("outputs are shorter than n_tasks")
+    _check(_load().infaas_autoscale_step(cat.handle, int(window_us), int(slack_pct), int(lambda_milli),
+                                         _dev_ptr(d_variant, "u32"), _dev_ptr(d_delta, "u32"),
+                                         _stream_ptr(stream)), "infaas_autoscale_step")
 
 
 def infaas_catalog_get_state(cat: Catalog, stream=None) -> dict:

@@ -18,6 +18,10 @@ struct infaas_catalog {
   std::vector<uint32_t> task_off, reg_off;
   uint32_t select_smem = 0;              // shared memory reserved for the staged image
   uint32_t worst_image_bytes = 0;        // image size if every block had its largest size
+  uint32_t *s_inst = nullptr;            // running instances per slot (Model-Autoscaler)
+  uint16_t *s_arch = nullptr;            // architecture code per slot
+  uint32_t *task_slo = nullptr;          // SLO per task
+  bool autoscale_ready = false;
 };
 
 namespace {
@@ -87,6 +91,7 @@ const char *infaas_strerror(int code) {
     case INFAAS_E_ALIGN: return "device array is not 16-byte aligned";
     case INFAAS_E_DEVICE: return "a kernel reported an internal error";
     case INFAAS_E_BAD_STATE: return "variant state is not one of INFAAS_STATE_*";
+    case INFAAS_E_BAD_ARG: return "a scalar argument is out of range, or a required set-up call is missing";
     default: return "unknown error code";
   }
 }
@@ -126,14 +131,14 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
 
   std::vector<uint32_t> h_lat(n_variants), h_cost(n_variants), h_id(n_variants), h_queued(n_variants),
       slot_of_id(n_variants);
-  std::vector<uint16_t> h_batch(n_variants), h_acc(n_variants);
+  std::vector<uint16_t> h_batch(n_variants), h_acc(n_variants), h_arch(n_variants);
   {
     std::vector<uint32_t> cursor(task_off.begin(), task_off.end() - 1);
     for (uint32_t v = 0; v < n_variants; ++v) {
       const infaas_variant &r = rows[v];
       const uint32_t s = cursor[r.task]++;
       h_lat[s] = r.lat_us; h_batch[s] = r.batch; h_acc[s] = r.acc_bp; h_cost[s] = r.cost;
-      h_id[s] = v; h_queued[s] = r.queued; slot_of_id[v] = s;
+      h_id[s] = v; h_queued[s] = r.queued; slot_of_id[v] = s; h_arch[s] = r.arch;
     }
   }
 
@@ -166,6 +171,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_pred = carve((size_t)n_variants * 4), o_served = carve((size_t)n_variants * 8);
   const size_t o_count = carve((size_t)n_variants * 4);
   const size_t o_state = carve((size_t)n_variants), o_load_lat = carve((size_t)n_variants * 4);
+  const size_t o_inst = carve((size_t)n_variants * 4), o_arch = carve((size_t)n_variants * 2);
+  const size_t o_task_slo = carve((size_t)n_tasks * 4);
   const size_t o_regions = carve((size_t)region_bytes);
   const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve(((size_t)n_tasks + n_extra) * 16);
   const size_t o_seg_base = carve((n_tasks + 1) * 4), o_xhdr = carve((size_t)n_extra * 16 + 16);
@@ -194,6 +201,10 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   LOAD_TRY(cudaMemcpy(base + o_cost, h_cost.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_id, h_id.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_queued, h_queued.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_arch, h_arch.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
+  c->s_inst = reinterpret_cast<uint32_t *>(base + o_inst);
+  c->s_arch = reinterpret_cast<uint16_t *>(base + o_arch);
+  c->task_slo = reinterpret_cast<uint32_t *>(base + o_task_slo);
 
   DeviceCatalog &d = c->d;
   d.n_variants = n_variants;
@@ -327,6 +338,33 @@ int infaas_catalog_get_states(infaas_catalog *c, uint8_t *h_state, void *cuda_st
   CUDA_TRY(cudaMemcpyAsync(st.data(), c->d.s_state, nv, cudaMemcpyDeviceToHost, s));
   CUDA_TRY(cudaStreamSynchronize(s));
   for (uint32_t v = 0; v < nv; ++v) h_state[v] = st[c->slot_of_id[v]];
+  return INFAAS_OK;
+}
+
+int infaas_autoscale_config(infaas_catalog *c, const uint32_t *h_instances, const uint32_t *h_task_slo_us,
+                            void *cuda_stream) {
+  if (!c || !h_instances || !h_task_slo_us) return INFAAS_E_NULL;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const uint32_t nv = c->d.n_variants;
+  std::vector<uint32_t> inst(nv);
+  for (uint32_t v = 0; v < nv; ++v) inst[c->slot_of_id[v]] = h_instances[v];
+  CUDA_TRY(cudaMemcpyAsync(c->s_inst, inst.data(), (size_t)nv * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(cudaMemcpyAsync(c->task_slo, h_task_slo_us, (size_t)c->d.n_tasks * 4, cudaMemcpyHostToDevice, s));
+  CUDA_TRY(cudaStreamSynchronize(s));
+  c->autoscale_ready = true;
+  return INFAAS_OK;
+}
+
+int infaas_autoscale_step(infaas_catalog *c, uint32_t window_us, uint32_t slack_pct, uint32_t lambda_milli,
+                          uint32_t *d_variant, uint32_t *d_delta, void *cuda_stream) {
+  if (!c || !d_variant || !d_delta) return INFAAS_E_NULL;
+  if (window_us == 0 || !c->autoscale_ready) return INFAAS_E_BAD_ARG;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  CUDA_TRY(infaas::launch_autoscale(c->d, c->s_inst, c->s_arch, c->task_slo, window_us, slack_pct, lambda_milli,
+                                    d_variant, d_delta, static_cast<cudaStream_t>(cuda_stream)));
   return INFAAS_OK;
 }
 
