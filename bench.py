@@ -318,6 +318,7 @@ def run_ours(args):
         if w.window and world == 1:
             out["windowed"] = windowed_leg(P, cat, w, inputs[0], d_dec, world)
             out["stateful"] = stateful_leg(P, w, inputs, d_dec, local, peak)
+            out["autoscale"] = autoscale_leg(P, w, inputs[0], d_dec, local)
     else:
         out["e2e"] = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -462,6 +463,57 @@ def stateful_leg(P, w, inputs, d_dec, local, peak):
             "states_after_windows": np.bincount(end, minlength=4).tolist(),
             "list_entries": info["list_entries"], "image_bytes": info["image_bytes"],
             "windowed_us_per_window": win["us_per_window"], "windowed_value": win["value"], "unit": UNIT}
+
+
+def autoscale_leg(P, w, inp, d_dec, local):
+    """Scaling-up step of the Model-Autoscaler on one window's tallies: every variant that
+    served queries in the window runs one instance, each task's SLO is the median SLO of its
+    queries, slack 1.05 (the paper's value), lambda 0.1/s.  One small kernel per window."""
+    import torch
+    from paper_1905_13348_b200 import workloads as W
+    t, s, a = inp
+    W_ = w.window
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks, local)
+    _, load = W.variant_states(w.n_variants)
+    P.infaas_catalog_set_states(cat, np.ones(w.n_variants, np.uint8), load)
+    P.infaas_select_batch(cat, t[:W_], s[:W_], a[:W_], d_dec[:W_])
+    P.infaas_tally(cat, d_dec[:W_])
+    torch.cuda.synchronize()
+    dec = d_dec[:W_].cpu().numpy().view(np.uint32)
+    served = np.bincount(dec[(dec >> 31) == 0], minlength=w.n_variants)
+    slo = np.array([np.median(w.slo_us[:W_][w.task[:W_] == k]) if (w.task[:W_] == k).any() else 0
+                    for k in range(w.n_tasks)], np.uint32)
+    P.infaas_autoscale_config(cat, (served > 0).astype(np.uint32), slo)
+    d_v = torch.empty(w.n_tasks, dtype=torch.int32, device="cuda")
+    d_d = torch.empty(w.n_tasks, dtype=torch.int32, device="cuda")
+    # 50 calls in one CUDA graph: the kernel is far shorter than a Python call
+    side = torch.cuda.Stream()
+    reps = 50
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            P.infaas_autoscale_step(cat, w.window_us, 105, 100, d_v, d_d, stream=side)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(reps):
+                P.infaas_autoscale_step(cat, w.window_us, 105, 100, d_v, d_d, stream=side)
+        graph.replay()
+        side.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        graph.replay()
+        e1.record(side)
+        side.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / reps
+    v = d_v.cpu().numpy().view(np.uint32)
+    d = d_d.cpu().numpy().view(np.uint32)
+    cat.free()
+    act = v < 0xFFFFFFFE
+    return {"us_per_step": us, "tasks": w.n_tasks, "window_queries": W_, "window_us": w.window_us,
+            "tasks_scaling": int(act.sum()), "tasks_with_headroom": int((v == 0xFFFFFFFF).sum()),
+            "tasks_escalated": int((v == 0xFFFFFFFE).sum()), "instances_added": int(d[act].sum()),
+            "how": "50 calls in one CUDA graph",
+            "bound": "latency (one CTA per task over ~30 B per variant)"}
 
 
 def main():

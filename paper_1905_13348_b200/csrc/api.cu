@@ -20,6 +20,7 @@ struct infaas_catalog {
   uint32_t worst_image_bytes = 0;        // image size if every block had its largest size
   uint32_t *s_inst = nullptr;            // running instances per slot (Model-Autoscaler)
   uint16_t *s_arch = nullptr;            // architecture code per slot
+  unsigned long long *s_qps = nullptr;   // profiled saturation throughput per slot, milli-queries/s
   uint32_t *task_slo = nullptr;          // SLO per task
   bool autoscale_ready = false;
 };
@@ -132,6 +133,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   std::vector<uint32_t> h_lat(n_variants), h_cost(n_variants), h_id(n_variants), h_queued(n_variants),
       slot_of_id(n_variants);
   std::vector<uint16_t> h_batch(n_variants), h_acc(n_variants), h_arch(n_variants);
+  std::vector<unsigned long long> h_qps(n_variants);
   {
     std::vector<uint32_t> cursor(task_off.begin(), task_off.end() - 1);
     for (uint32_t v = 0; v < n_variants; ++v) {
@@ -139,6 +141,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
       const uint32_t s = cursor[r.task]++;
       h_lat[s] = r.lat_us; h_batch[s] = r.batch; h_acc[s] = r.acc_bp; h_cost[s] = r.cost;
       h_id[s] = v; h_queued[s] = r.queued; slot_of_id[v] = s; h_arch[s] = r.arch;
+      h_qps[s] = 1000000000ull * r.batch / r.lat_us;     // floor(10^9 * batch / lat_us)
     }
   }
 
@@ -172,7 +175,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_count = carve((size_t)n_variants * 4);
   const size_t o_state = carve((size_t)n_variants), o_load_lat = carve((size_t)n_variants * 4);
   const size_t o_inst = carve((size_t)n_variants * 4), o_arch = carve((size_t)n_variants * 2);
-  const size_t o_task_slo = carve((size_t)n_tasks * 4);
+  const size_t o_task_slo = carve((size_t)n_tasks * 4), o_qps = carve((size_t)n_variants * 8);
   const size_t o_regions = carve((size_t)region_bytes);
   const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve(((size_t)n_tasks + n_extra) * 16);
   const size_t o_seg_base = carve((n_tasks + 1) * 4), o_xhdr = carve((size_t)n_extra * 16 + 16);
@@ -202,6 +205,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   LOAD_TRY(cudaMemcpy(base + o_id, h_id.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_queued, h_queued.data(), (size_t)n_variants * 4, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_arch, h_arch.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
+  LOAD_TRY(cudaMemcpy(base + o_qps, h_qps.data(), (size_t)n_variants * 8, cudaMemcpyHostToDevice));
+  c->s_qps = reinterpret_cast<unsigned long long *>(base + o_qps);
   c->s_inst = reinterpret_cast<uint32_t *>(base + o_inst);
   c->s_arch = reinterpret_cast<uint16_t *>(base + o_arch);
   c->task_slo = reinterpret_cast<uint32_t *>(base + o_task_slo);
@@ -363,7 +368,7 @@ int infaas_autoscale_step(infaas_catalog *c, uint32_t window_us, uint32_t slack_
   if (window_us == 0 || !c->autoscale_ready) return INFAAS_E_BAD_ARG;
   DeviceScope scope(c->device);
   if (scope.status != cudaSuccess) return cuda_fail(scope.status);
-  CUDA_TRY(infaas::launch_autoscale(c->d, c->s_inst, c->s_arch, c->task_slo, window_us, slack_pct, lambda_milli,
+  CUDA_TRY(infaas::launch_autoscale(c->d, c->s_inst, c->s_arch, c->s_qps, c->task_slo, window_us, slack_pct, lambda_milli,
                                     d_variant, d_delta, static_cast<cudaStream_t>(cuda_stream)));
   return INFAAS_OK;
 }

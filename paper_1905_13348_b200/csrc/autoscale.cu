@@ -19,10 +19,6 @@ __device__ __forceinline__ unsigned long long sat_add(unsigned long long a, unsi
 __device__ __forceinline__ unsigned long long sat_mul(unsigned long long a, unsigned long long b) {
   return __umul64hi(a, b) ? U64_MAX_ : a * b;
 }
-// Saturation throughput in milli-queries per second.
-__device__ __forceinline__ unsigned long long sat_qps(uint32_t batch, uint32_t lat_us) {
-  return 1000000000ull * batch / lat_us;
-}
 // ceil(x * m / 100), saturating at 2^64-1.
 __device__ unsigned long long scale_pct_ceil(unsigned long long x, uint32_t m) {
   unsigned long long hi = __umul64hi(x, (unsigned long long)m), lo = x * m;
@@ -51,7 +47,8 @@ __device__ __forceinline__ bool better(const Action &a, const Action &b) {
 }
 
 __global__ void __launch_bounds__(AUTOSCALE_THREADS)
-autoscale_kernel(DeviceCatalog c, const uint32_t *s_inst, const uint16_t *s_arch, const uint32_t *task_slo,
+autoscale_kernel(DeviceCatalog c, const uint32_t *s_inst, const uint16_t *s_arch,
+                 const unsigned long long *s_qps, const uint32_t *task_slo,
                  uint32_t window_us, uint32_t slack_pct, uint32_t lambda_milli, uint32_t *out_variant,
                  uint32_t *out_delta) {
   __shared__ unsigned long long w_served[AUTOSCALE_THREADS / 32], w_cap[AUTOSCALE_THREADS / 32],
@@ -70,7 +67,7 @@ autoscale_kernel(DeviceCatalog c, const uint32_t *s_inst, const uint16_t *s_arch
     const uint32_t id = c.s_id[s], cnt = c.count_by_id[id], n = s_inst[s];
     served += cnt;
     if (n) {
-      cap = sat_add(cap, sat_mul(n, sat_qps(c.s_batch[s], c.s_lat[s])));
+      cap = sat_add(cap, sat_mul(n, s_qps[s]));
       const unsigned long long k = ((unsigned long long)cnt << 32) | (0xFFFFFFFFu - id);
       if (k > key) { key = k; key_slot = s; }
     }
@@ -106,13 +103,13 @@ autoscale_kernel(DeviceCatalog c, const uint32_t *s_inst, const uint16_t *s_arch
   const uint32_t r = s_r, slo = task_slo[t];
   unsigned long long q_r = 0;
   uint32_t arch_r = 0;
-  if (r != 0xFFFFFFFFu) { q_r = sat_qps(c.s_batch[r], c.s_lat[r]); arch_r = s_arch[r]; }
+  if (r != 0xFFFFFFFFu) { q_r = s_qps[r]; arch_r = s_arch[r]; }
 
   Action best;
   best.id = 0xFFFFFFFFu; best.cost_hi = best.cost_lo = 0; best.kind = 0; best.delta = 0;
   for (uint32_t s = lo + tid; s < hi; s += AUTOSCALE_THREADS) {
     const uint32_t lat = c.s_lat[s];
-    const unsigned long long q = sat_qps(c.s_batch[s], lat);
+    const unsigned long long q = s_qps[s];               // saturation throughput, milli-queries/s
     if (q == 0ull || lat > slo) continue;         // constraint (2): new instances meet the SLO
     uint32_t kind = 1;                             // 0 replicate, 1 upgrade
     if (s == r) kind = 0;
@@ -149,10 +146,10 @@ autoscale_kernel(DeviceCatalog c, const uint32_t *s_inst, const uint16_t *s_arch
 }  // namespace
 
 cudaError_t launch_autoscale(const DeviceCatalog &c, const uint32_t *s_inst, const uint16_t *s_arch,
-                             const uint32_t *task_slo, uint32_t window_us, uint32_t slack_pct,
+                             const unsigned long long *s_qps, const uint32_t *task_slo, uint32_t window_us, uint32_t slack_pct,
                              uint32_t lambda_milli, uint32_t *d_variant, uint32_t *d_delta,
                              cudaStream_t stream) {
-  autoscale_kernel<<<c.n_tasks, AUTOSCALE_THREADS, 0, stream>>>(c, s_inst, s_arch, task_slo, window_us, slack_pct,
+  autoscale_kernel<<<c.n_tasks, AUTOSCALE_THREADS, 0, stream>>>(c, s_inst, s_arch, s_qps, task_slo, window_us, slack_pct,
                                                                 lambda_milli, d_variant, d_delta);
   return cudaGetLastError();
 }

@@ -211,9 +211,10 @@ cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const 
                           int sm_count, uint32_t image_smem, cudaStream_t stream);
 
 // Scaling-up step of the Model-Autoscaler for every task, from the pending per-variant
-// counts; s_inst / s_arch are per slot, task_slo per task; outputs have n_tasks entries.
+// counts; s_inst / s_arch / s_qps (floor(10^9 * batch / lat_us)) are per slot, task_slo per
+// task; outputs have n_tasks entries.
 cudaError_t launch_autoscale(const DeviceCatalog &c, const uint32_t *s_inst, const uint16_t *s_arch,
-                             const uint32_t *task_slo, uint32_t window_us, uint32_t slack_pct,
+                             const unsigned long long *s_qps, const uint32_t *task_slo, uint32_t window_us, uint32_t slack_pct,
                              uint32_t lambda_milli, uint32_t *d_variant, uint32_t *d_delta,
                              cudaStream_t stream);
 
