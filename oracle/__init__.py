@@ -1,3 +1,4 @@
 """CPU oracle (test infrastructure only; never imported by the CUDA path)."""
 from .oracle import (ACTIVE, AUTOSCALE_ESCALATE, AUTOSCALE_NONE, INACTIVE, INTERFERED,  # noqa: F401
-                     OVERLOADED, OracleCatalog, StatefulOracleCatalog, autoscale_step, build, pred_lat)
+                     OVERLOADED, OracleCatalog, StatefulOracleCatalog, assign_workers, autoscale_step,
+                     build, pred_lat)

@@ -27,6 +27,9 @@
 //     replicating the running variant and upgrading to a faster one of the same architecture
 //     (Section 4.2.1 cost function and constraints; Section 4.2.2 scaling-up algorithm).
 //
+//   * The query is sent to the least-loaded worker that runs the chosen variant, or, if the
+//     variant is not loaded, to the least-utilised worker with its hardware (Section 4.1).
+//
 // Everything is brute force over the full, unsorted, unpruned catalog.  There is no
 // sorting, no pruning, no early exit and no blocking.  Readings of points the paper leaves
 // open (ties, the queueing term, the distance used for "closest", the queue recursion, what
@@ -376,6 +379,41 @@ void oracle_autoscale_step(const void *rows_v, uint32_t n_variants, uint32_t n_t
     }
     action_variant[t] = have_best ? best_v : AUTOSCALE_ESCALATE;
     action_delta[t] = have_best ? best_delta : 0;
+  }
+}
+
+// ---- worker choice (Section 4.1, Case I: the Active variant's query goes to the least-loaded
+// worker running an instance of it, an Inactive variant's to the worker with the lowest
+// utilisation on the variant's target hardware; Section 5: an instance is a {variant, worker}
+// pair) ----
+// Per query with a feasible decision v (bit 31 clear, v < n_variants), against one snapshot:
+//   some instance of v exists: the worker of the instance with the smallest (load, worker);
+//   else: the worker with the smallest (util, worker index) among workers whose hardware code
+//   equals hw(v); none: 0xFFFFFFFF.  Other decisions: 0xFFFFFFFF.
+void oracle_assign_workers(const void *rows_v, uint32_t n_variants, const uint32_t *inst_variant,
+                           const uint32_t *inst_worker, const uint32_t *inst_load, uint32_t n_inst,
+                           const uint8_t *worker_hw, const uint32_t *worker_util, uint32_t n_workers,
+                           const uint32_t *decision, uint64_t n, uint32_t *worker) {
+  const Row *rows = (const Row *)rows_v;
+  for (uint64_t q = 0; q < n; ++q) {
+    uint32_t v = decision[q];
+    worker[q] = INVALID;
+    if ((v & NO_FEASIBLE_BIT) || v >= n_variants) continue;
+    bool have = false;
+    uint64_t best_load = 0, best_w = 0;
+    for (uint32_t i = 0; i < n_inst; ++i) {
+      if (inst_variant[i] != v || inst_worker[i] >= n_workers) continue;
+      if (!have || inst_load[i] < best_load || (inst_load[i] == best_load && inst_worker[i] < best_w)) {
+        have = true; best_load = inst_load[i]; best_w = inst_worker[i];
+      }
+    }
+    if (!have) {
+      for (uint32_t w = 0; w < n_workers; ++w) {
+        if (worker_hw[w] != rows[v].hw) continue;
+        if (!have || worker_util[w] < best_load) { have = true; best_load = worker_util[w]; best_w = w; }
+      }
+    }
+    if (have) worker[q] = (uint32_t)best_w;
   }
 }
 

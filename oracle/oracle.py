@@ -64,6 +64,10 @@ def _load():
         lib.oracle_autoscale_step.restype = None
         lib.oracle_autoscale_step.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32] + \
             [ctypes.c_void_p] * 4 + [ctypes.c_uint32] * 3 + [ctypes.c_void_p] * 2
+        lib.oracle_assign_workers.restype = None
+        lib.oracle_assign_workers.argtypes = [ctypes.c_void_p, ctypes.c_uint32] + [ctypes.c_void_p] * 3 + \
+            [ctypes.c_uint32] + [ctypes.c_void_p] * 2 + [ctypes.c_uint32, ctypes.c_void_p, ctypes.c_uint64,
+                                                         ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -160,3 +164,18 @@ def autoscale_step(rows: np.ndarray, n_tasks: int, count, instances, load_lat_us
                                   _ptr(task_slo_us), int(window_us), int(slack_pct), int(lambda_milli),
                                   _ptr(variant), _ptr(delta))
     return variant, delta
+
+
+def assign_workers(rows: np.ndarray, inst_variant, inst_worker, inst_load, worker_hw, worker_util, decision):
+    """Worker for every decision against one snapshot of the instance and worker tables
+    (Section 4.1, Case I); see oracle_assign_workers in infaas_oracle.cpp."""
+    rows = np.ascontiguousarray(rows)
+    iv, iw, il = (np.ascontiguousarray(a, np.uint32) for a in (inst_variant, inst_worker, inst_load))
+    hw = np.ascontiguousarray(worker_hw, np.uint8)
+    ut = np.ascontiguousarray(worker_util, np.uint32)
+    decision = np.ascontiguousarray(decision, np.uint32)
+    assert iv.shape == iw.shape == il.shape and hw.shape == ut.shape
+    out = np.empty(decision.shape[0], np.uint32)
+    _load().oracle_assign_workers(_ptr(rows), rows.shape[0], _ptr(iv), _ptr(iw), _ptr(il), iv.shape[0],
+                                  _ptr(hw), _ptr(ut), hw.shape[0], _ptr(decision), decision.shape[0], _ptr(out))
+    return out
