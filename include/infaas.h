@@ -216,6 +216,31 @@ int infaas_autoscale_step(infaas_catalog *c, uint32_t window_us, uint32_t slack_
                           uint32_t lambda_milli, uint32_t *d_variant, uint32_t *d_delta,
                           void *cuda_stream);
 
+/* Worker choice (Section 4.1, Case I; Section 5: an instance is a {variant, worker} pair).  A
+ * decided query goes to the least-loaded worker that runs an instance of the chosen variant;
+ * if the variant is not loaded anywhere, to the worker with the lowest utilisation among those
+ * whose hardware is the variant's (the row's hw code).  All queries of a call see one snapshot
+ * of the two tables:
+ *     worker(q) = the worker of the instance of v = d_decision[q] with the smallest
+ *                 (load, worker);  if v has no instance, the w with the smallest (util, w) among
+ *                 worker_hw[w] == hw(v);  if there is none, or the decision has bit 31 set or is
+ *                 >= n_variants, 0xFFFFFFFF.
+ *   infaas_workers_config: HOST arrays, copied: the instance table h_inst_variant /
+ *     h_inst_worker / h_inst_load (n_inst entries each; rows whose variant or worker is out of
+ *     range are ignored; may be NULL if n_inst == 0) and the worker table h_worker_hw (u8) /
+ *     h_worker_util (n_workers entries; worker ids are the indices).  Replaces the previous
+ *     tables (the paper's monitoring daemons refresh them every 2 s).  Allocates and frees a
+ *     temporary device buffer; synchronises cuda_stream.  Errors: E_NULL, E_CUDA.
+ *   infaas_assign_workers: d_decision DEVICE n u32 (read), d_worker DEVICE n u32 (written),
+ *     both 16-byte aligned; asynchronous, stream-ordered, allocates nothing.  Errors: E_NULL,
+ *     E_ALIGN, E_BAD_ARG (infaas_workers_config never called), E_CUDA. */
+int infaas_workers_config(infaas_catalog *c, const uint32_t *h_inst_variant,
+                          const uint32_t *h_inst_worker, const uint32_t *h_inst_load,
+                          uint32_t n_inst, const uint8_t *h_worker_hw,
+                          const uint32_t *h_worker_util, uint32_t n_workers, void *cuda_stream);
+int infaas_assign_workers(infaas_catalog *c, const uint32_t *d_decision, uint64_t n,
+                          uint32_t *d_worker, void *cuda_stream);
+
 /* Copy the load state to HOST arrays (any of the four may be NULL to skip it):
  *   h_queued[n_variants], h_pred_lat_us[n_variants], h_served_total[n_variants] indexed by
  *   variant id; h_counters[3] = feasible decisions tallied, NO_FEASIBLE decisions seen,

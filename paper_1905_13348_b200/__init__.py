@@ -10,7 +10,7 @@ _BINDING = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
             "infaas_tally", "infaas_pending_counts", "infaas_advance", "infaas_catalog_set_states",
             "infaas_catalog_get_states", "STATE_INACTIVE", "STATE_ACTIVE", "STATE_OVERLOADED",
             "STATE_INTERFERED", "infaas_autoscale_config", "infaas_autoscale_step", "AUTOSCALE_NONE",
-            "AUTOSCALE_ESCALATE", "Catalog", "InfaasError",
+            "AUTOSCALE_ESCALATE", "infaas_workers_config", "infaas_assign_workers", "Catalog", "InfaasError",
             "NO_FEASIBLE", "INVALID")
 
 

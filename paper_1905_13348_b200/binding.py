@@ -26,7 +26,8 @@ EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info",
            "infaas_tally", "infaas_pending_counts", "infaas_advance",
            "infaas_catalog_set_states", "infaas_catalog_get_states",
-           "infaas_autoscale_config", "infaas_autoscale_step")
+           "infaas_autoscale_config", "infaas_autoscale_step",
+           "infaas_workers_config", "infaas_assign_workers")
 
 
 class InfaasError(RuntimeError):
@@ -70,6 +71,9 @@ def _load():
     lib.infaas_autoscale_config.argtypes = [vp, vp, vp, vp]
     lib.infaas_autoscale_step.argtypes = [vp, u32, u32, u32, vp, vp, vp]
     lib.infaas_autoscale_config.restype = lib.infaas_autoscale_step.restype = i32
+    lib.infaas_workers_config.argtypes = [vp, vp, vp, vp, u32, vp, vp, u32, vp]
+    lib.infaas_assign_workers.argtypes = [vp, vp, u64, vp, vp]
+    lib.infaas_workers_config.restype = lib.infaas_assign_workers.restype = i32
     lib.infaas_tally_static.argtypes = [vp, u64, u32, vp, vp, i32, vp]
     lib.infaas_tally_static.restype = i32
     lib.infaas_strerror.argtypes = [i32]
@@ -204,6 +208,26 @@ def infaas_autoscale_step(cat: Catalog, window_us: int, slack_pct: int, lambda_m
     _check(_load().infaas_autoscale_step(cat.handle, int(window_us), int(slack_pct), int(lambda_milli),
                                          _dev_ptr(d_variant, "u32"), _dev_ptr(d_delta, "u32"),
                                          _stream_ptr(stream)), "infaas_autoscale_step")
+
+
+def infaas_workers_config(cat: Catalog, inst_variant, inst_worker, inst_load, worker_hw, worker_util,
+                          stream=None) -> None:
+    """Host arrays: the instance table (three u32 arrays of equal length) and the worker table
+    (u8 hardware codes, u32 utilisations; worker id = index)."""
+    iv, iw, il = (np.ascontiguousarray(a, np.uint32) for a in (inst_variant, inst_worker, inst_load))
+    hw = np.ascontiguousarray(worker_hw, np.uint8)
+    ut = np.ascontiguousarray(worker_util, np.uint32)
+    if not (iv.shape == iw.shape == il.shape and iv.ndim == 1 and hw.shape == ut.shape and hw.ndim == 1):
+        raise ValueError("instance arrays must have one length, worker arrays another")
+    p = lambda a: a.ctypes.data if a.size else None
+    _check(_load().infaas_workers_config(cat.handle, p(iv), p(iw), p(il), iv.shape[0], p(hw), p(ut), hw.shape[0],
+                                         _stream_ptr(stream)), "infaas_workers_config")
+
+
+def infaas_assign_workers(cat: Catalog, d_decision, d_worker, n=None, stream=None) -> None:
+    n = int(d_decision.shape[0]) if n is None else int(n)
+    _check(_load().infaas_assign_workers(cat.handle, _dev_ptr(d_decision, "u32"), n, _dev_ptr(d_worker, "u32"),
+                                         _stream_ptr(stream)), "infaas_assign_workers")
 
 
 def infaas_catalog_get_state(cat: Catalog, stream=None) -> dict:

@@ -23,6 +23,10 @@ struct infaas_catalog {
   unsigned long long *s_qps = nullptr;   // profiled saturation throughput per slot, milli-queries/s
   uint32_t *task_slo = nullptr;          // SLO per task
   bool autoscale_ready = false;
+  unsigned char *hw_by_id = nullptr;     // hardware code per variant id (worker choice)
+  uint32_t *worker_of = nullptr;         // worker per variant id
+  unsigned long long *best_inst = nullptr, *best_hw = nullptr;   // scratch of the table build
+  bool workers_ready = false;
 };
 
 namespace {
@@ -176,6 +180,8 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   const size_t o_state = carve((size_t)n_variants), o_load_lat = carve((size_t)n_variants * 4);
   const size_t o_inst = carve((size_t)n_variants * 4), o_arch = carve((size_t)n_variants * 2);
   const size_t o_task_slo = carve((size_t)n_tasks * 4), o_qps = carve((size_t)n_variants * 8);
+  const size_t o_hw = carve((size_t)n_variants), o_worker_of = carve((size_t)n_variants * 4);
+  const size_t o_best_inst = carve((size_t)n_variants * 8), o_best_hw = carve(256 * 8);
   const size_t o_regions = carve((size_t)region_bytes);
   const size_t o_flen = carve((size_t)n_tasks * 4), o_slow = carve(((size_t)n_tasks + n_extra) * 16);
   const size_t o_seg_base = carve((n_tasks + 1) * 4), o_xhdr = carve((size_t)n_extra * 16 + 16);
@@ -207,6 +213,15 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   LOAD_TRY(cudaMemcpy(base + o_arch, h_arch.data(), (size_t)n_variants * 2, cudaMemcpyHostToDevice));
   LOAD_TRY(cudaMemcpy(base + o_qps, h_qps.data(), (size_t)n_variants * 8, cudaMemcpyHostToDevice));
   c->s_qps = reinterpret_cast<unsigned long long *>(base + o_qps);
+  {
+    std::vector<unsigned char> h_hw(n_variants);
+    for (uint32_t v = 0; v < n_variants; ++v) h_hw[v] = rows[v].hw;
+    LOAD_TRY(cudaMemcpy(base + o_hw, h_hw.data(), n_variants, cudaMemcpyHostToDevice));
+  }
+  c->hw_by_id = base + o_hw;
+  c->worker_of = reinterpret_cast<uint32_t *>(base + o_worker_of);
+  c->best_inst = reinterpret_cast<unsigned long long *>(base + o_best_inst);
+  c->best_hw = reinterpret_cast<unsigned long long *>(base + o_best_hw);
   c->s_inst = reinterpret_cast<uint32_t *>(base + o_inst);
   c->s_arch = reinterpret_cast<uint16_t *>(base + o_arch);
   c->task_slo = reinterpret_cast<uint32_t *>(base + o_task_slo);
@@ -370,6 +385,55 @@ int infaas_autoscale_step(infaas_catalog *c, uint32_t window_us, uint32_t slack_
   if (scope.status != cudaSuccess) return cuda_fail(scope.status);
   CUDA_TRY(infaas::launch_autoscale(c->d, c->s_inst, c->s_arch, c->s_qps, c->task_slo, window_us, slack_pct, lambda_milli,
                                     d_variant, d_delta, static_cast<cudaStream_t>(cuda_stream)));
+  return INFAAS_OK;
+}
+
+int infaas_workers_config(infaas_catalog *c, const uint32_t *h_inst_variant, const uint32_t *h_inst_worker,
+                          const uint32_t *h_inst_load, uint32_t n_inst, const uint8_t *h_worker_hw,
+                          const uint32_t *h_worker_util, uint32_t n_workers, void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  if (n_inst && (!h_inst_variant || !h_inst_worker || !h_inst_load)) return INFAAS_E_NULL;
+  if (n_workers && (!h_worker_hw || !h_worker_util)) return INFAAS_E_NULL;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  // one temporary buffer: three u32 arrays of n_inst, one u32 array and one u8 array of n_workers
+  const size_t ib = round_up((size_t)n_inst * 4, 256), wb = round_up((size_t)n_workers * 4, 256);
+  unsigned char *tmp = nullptr;
+  CUDA_TRY(cudaMalloc(&tmp, 3 * ib + 2 * wb + 256));
+  uint32_t *d_iv = reinterpret_cast<uint32_t *>(tmp), *d_iw = reinterpret_cast<uint32_t *>(tmp + ib),
+           *d_il = reinterpret_cast<uint32_t *>(tmp + 2 * ib), *d_wu = reinterpret_cast<uint32_t *>(tmp + 3 * ib);
+  unsigned char *d_wh = tmp + 3 * ib + wb;
+  cudaError_t e = cudaSuccess;
+  auto up = [&](void *dst, const void *src, size_t bytes) {
+    if (e == cudaSuccess && bytes) e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyHostToDevice, s);
+  };
+  up(d_iv, h_inst_variant, (size_t)n_inst * 4);
+  up(d_iw, h_inst_worker, (size_t)n_inst * 4);
+  up(d_il, h_inst_load, (size_t)n_inst * 4);
+  up(d_wu, h_worker_util, (size_t)n_workers * 4);
+  up(d_wh, h_worker_hw, (size_t)n_workers);
+  if (e == cudaSuccess)
+    e = infaas::launch_workers_build(c->d.n_variants, c->hw_by_id, d_iv, d_iw, d_il, n_inst, d_wh, d_wu, n_workers,
+                                     c->best_inst, c->best_hw, c->worker_of, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  (void)cudaFree(tmp);
+  if (e != cudaSuccess) return cuda_fail(e);
+  c->workers_ready = true;
+  return INFAAS_OK;
+}
+
+int infaas_assign_workers(infaas_catalog *c, const uint32_t *d_decision, uint64_t n, uint32_t *d_worker,
+                          void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  if (!c->workers_ready) return INFAAS_E_BAD_ARG;
+  if (n == 0) return INFAAS_OK;
+  if (!d_decision || !d_worker) return INFAAS_E_NULL;
+  if (!aligned16(d_decision) || !aligned16(d_worker)) return INFAAS_E_ALIGN;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  CUDA_TRY(infaas::launch_assign_workers(d_decision, n, c->d.n_variants, c->worker_of, d_worker, c->sm_count,
+                                         static_cast<cudaStream_t>(cuda_stream)));
   return INFAAS_OK;
 }
 

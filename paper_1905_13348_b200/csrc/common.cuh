@@ -218,4 +218,18 @@ cudaError_t launch_autoscale(const DeviceCatalog &c, const uint32_t *s_inst, con
                              uint32_t lambda_milli, uint32_t *d_variant, uint32_t *d_delta,
                              cudaStream_t stream);
 
+// Worker choice.  Build: one worker per variant from the instance table {variant, worker, load}
+// and the worker table {hardware code, utilisation} (device arrays); best_inst [n_variants] and
+// best_hw [256] are scratch.  Assign: worker[q] = worker_of[decision[q]] for decisions below
+// n_variants, INFAAS_INVALID otherwise.
+cudaError_t launch_workers_build(uint32_t n_variants, const unsigned char *hw_by_id,
+                                 const uint32_t *inst_variant, const uint32_t *inst_worker,
+                                 const uint32_t *inst_load, uint32_t n_inst, const unsigned char *worker_hw,
+                                 const uint32_t *worker_util, uint32_t n_workers,
+                                 unsigned long long *best_inst, unsigned long long *best_hw,
+                                 uint32_t *worker_of, cudaStream_t stream);
+cudaError_t launch_assign_workers(const uint32_t *d_decision, uint64_t n, uint32_t n_variants,
+                                  const uint32_t *worker_of, uint32_t *d_worker, int sm_count,
+                                  cudaStream_t stream);
+
 }  // namespace infaas

@@ -27,6 +27,8 @@ def plain(rows, iv, iw, il, hw, ut, d):
 def test_against_sorting(seed):
     rng = np.random.default_rng(400 + seed)
     nv, nw, ni = int(rng.integers(1, 12)), int(rng.integers(1, 7)), int(rng.integers(0, 25))
+    if seed % 2:
+        nv, nw, ni = int(rng.integers(1, 4)), int(rng.integers(3, 9)), 40      # many instances per variant
     rows = _rows(nv, rng.integers(0, 3, nv))
     iv, iw = rng.integers(0, nv + 1, ni), rng.integers(0, nw + 1, ni)     # some rows point nowhere
     il = rng.integers(0, 4, ni)                                          # many equal loads
