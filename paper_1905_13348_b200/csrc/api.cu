@@ -71,7 +71,7 @@ inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // refreshes without a change of plan), none for the image if it does not -- the kernel
 // then reads it from global memory and the space is worth more as L1 cache.
 int refresh_select_plan(infaas_catalog *c, cudaStream_t stream) {
-  uint32_t hdr[4] = {0, 0, 0, 0};
+  uint32_t hdr[1] = {0};
   CUDA_TRY(cudaMemcpyAsync(hdr, c->d.image_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, stream));
   CUDA_TRY(cudaStreamSynchronize(stream));
   const uint32_t room = infaas::select_image_smem(infaas::SELECT_MAX_SMEM);
@@ -253,7 +253,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.image_capacity = (uint32_t)worst_image;
   d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
   d.counters = reinterpret_cast<unsigned long long *>(base + o_counters);
-  d.rebuild_ctr = reinterpret_cast<uint32_t *>(base + o_rebuild);
+  d.alloc_ctr = reinterpret_cast<unsigned long long *>(base + o_rebuild);
   d.err = reinterpret_cast<uint32_t *>(base + o_err);
   d.slo_seen = reinterpret_cast<uint32_t *>(base + o_seen);
   c->slot_of_id.swap(slot_of_id);
@@ -509,10 +509,23 @@ int infaas_catalog_get_info(infaas_catalog *c, uint32_t h_info[8], void *cuda_st
   DeviceScope scope(c->device);
   if (scope.status != cudaSuccess) return cuda_fail(scope.status);
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  uint32_t hdr[4] = {0, 0, 0, 0};
-  CUDA_TRY(cudaMemcpyAsync(hdr, c->d.image_hdr, sizeof(hdr), cudaMemcpyDeviceToHost, s));
+  // the image size comes from the rebuild kernel; the list statistics are summed up here
+  // from the per-task lengths and flags (reporting only)
+  const uint32_t T = c->d.n_tasks;
+  uint32_t bytes = 0;
+  std::vector<uint32_t> f_len(T);
+  std::vector<uint4> slow(T);
+  CUDA_TRY(cudaMemcpyAsync(&bytes, c->d.image_hdr, 4, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaMemcpyAsync(f_len.data(), c->d.f_len, (size_t)T * 4, cudaMemcpyDeviceToHost, s));
+  CUDA_TRY(cudaMemcpyAsync(slow.data(), c->d.slow, (size_t)T * 16, cudaMemcpyDeviceToHost, s));
   CUDA_TRY(cudaStreamSynchronize(s));
-  for (int i = 0; i < 4; ++i) h_info[i] = hdr[i];
+  h_info[0] = bytes;
+  h_info[1] = h_info[2] = h_info[3] = 0;
+  for (uint32_t t = 0; t < T; ++t) {
+    if (f_len[t] > h_info[1]) h_info[1] = f_len[t];
+    h_info[2] += f_len[t];
+    if (f_len[t] > 0 && (slow[t].z & infaas::TASK_FLAG_NOT_INDEXED)) ++h_info[3];
+  }
   h_info[4] = infaas::select_image_smem(c->select_smem);
   h_info[5] = h_info[6] = h_info[7] = 0;
   return INFAAS_OK;

@@ -69,7 +69,8 @@ namespace infaas {
 //
 // Per task in global memory (`regions`): keys u64[V] (pred_lat | acc_bp << 32, scan order,
 // F used; for Inactive entries the latency includes the loading latency) and ids u32[V], for
-// lists without an index and for inspection.
+// lists without an index and for inspection; then local u16[V], the entries' indices inside
+// the task, which the next rebuild uses as its first filter.
 // ---------------------------------------------------------------------------------------
 constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
@@ -134,7 +135,7 @@ inline __host__ __device__ uint32_t block_capacity(uint32_t V) {
   const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
   return block_layout(F, F, F, MAX_ACC_WORDS).bytes;
 }
-inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_up_u32(12u * V, 64u); }
+inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_up_u32(14u * V, 64u); }
 
 // Slow-path parameters of a list segment (one uint4 each, global memory; a task's first
 // segment at index task, further segments at n_tasks + their index).
@@ -172,10 +173,11 @@ struct DeviceCatalog {
 
   unsigned char *image;      // packed image, image_capacity bytes, 256-byte aligned
   uint32_t image_capacity;
-  uint32_t *image_hdr;       // [4]: bytes, longest list, total entries, tasks not indexed
+  uint32_t *image_hdr;       // [0]: bytes of the image (published by the rebuild kernel)
 
   unsigned long long *counters;  // [3] feasible, no-feasible, invalid
-  uint32_t *rebuild_ctr;         // [4] CTA arrival counter, block cursor, longest, entries (rebuild kernel)
+  unsigned long long *alloc_ctr; // rebuild kernel: block cursor (low 32 bits) | CTAs done allocating << 32;
+                                 // zero between kernels
   uint32_t *err;                 // sticky device error word (0 = fine)
   uint32_t *slo_seen;            // OR of all SLOs the selection kernel has read
 };

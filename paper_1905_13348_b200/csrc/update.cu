@@ -209,6 +209,19 @@ __device__ __forceinline__ uint32_t group8_or(uint32_t v) {
   return v;
 }
 
+// One atomic per allocation places a block in the image and, on a CTA's last allocation
+// (`done`), counts the CTA as finished with the cursor.  The CTA that is counted last knows the
+// final image size: it publishes it for the kernels that follow and clears the counter for the
+// next rebuild.  Thread 0 only; returns the block's offset behind the fixed part of the image.
+__device__ __forceinline__ uint32_t place_block(const DeviceCatalog &c, uint32_t bytes, bool done) {
+  const unsigned long long old = atomicAdd(c.alloc_ctr, ((unsigned long long)(done ? 1u : 0u) << 32) | bytes);
+  if (done && (uint32_t)(old >> 32) == gridDim.x - 1u) {
+    c.image_hdr[0] = image_var_offset(c.n_tasks) + (uint32_t)old + bytes;
+    *c.alloc_ctr = 0ull;
+  }
+  return (uint32_t)old;
+}
+
 // Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh) into
 // a block of the image obtained from the block cursor.  S.pred / S.acc / S.ids hold the
 // list in scan order.  Returns false (all threads) if the list cannot be indexed: its
@@ -217,7 +230,8 @@ __device__ __forceinline__ uint32_t group8_or(uint32_t v) {
 // the tables, which do not depend on each other, are written by different groups of warps.
 // `xi`: 0xFFFFFFFF for the task's first segment (header and SLO records go into the image), else
 // the index of this further segment (header to xhdr[xi], no records: only the slow path comes
-// here).  `next`: 1 + index of the task's next segment, 0 if this is the last.
+// here).  `next`: 1 + index of the task's next segment, 0 if this is the last (the CTA's last
+// allocation, then).
 __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, IndexScratch &S, uint32_t xi,
                             uint32_t next) {
   const uint32_t tid = threadIdx.x, B = blockDim.x;
@@ -298,11 +312,9 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   const BlockLayout BL = block_layout(F, Ks, Ka, nbw);
   const SlowLayout SL = slow_layout(F, Ks, Ka);
   if (tid == 0) {
-    uint32_t base = 0xFFFFFFFFu;
-    if (nbw <= MAX_ACC_WORDS) {
-      base = image_var_offset(c.n_tasks) + atomicAdd(&c.rebuild_ctr[1], BL.bytes);
-      if (base + BL.bytes > c.image_capacity || base + BL.t2 >= IMAGE_T2_LIMIT) base = 0xFFFFFFFFu;
-    }
+    const bool fits = nbw <= MAX_ACC_WORDS;
+    uint32_t base = image_var_offset(c.n_tasks) + place_block(c, fits ? BL.bytes : 0u, next == 0u);
+    if (!fits || base + BL.bytes > c.image_capacity || base + BL.t2 >= IMAGE_T2_LIMIT) base = 0xFFFFFFFFu;
     S.base = base;
   }
   __syncthreads();
@@ -418,7 +430,8 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
   unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
-  __shared__ uint32_t s_last, s_total, s_inlist;
+  __shared__ uint32_t s_total, s_inlist, s_ncand;
+  __shared__ uint16_t filt[RANK_SORT_MAX], cand[RANK_SORT_MAX];   // small tasks: filter set, candidates
   __shared__ IndexScratch S;
 
   const uint32_t t = blockIdx.x, tid = threadIdx.x, B = blockDim.x;
@@ -442,11 +455,15 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   unsigned char *region = c.regions + c.reg_off[t];
   unsigned long long *keys_g = reinterpret_cast<unsigned long long *>(region);
   uint32_t *ids_g = reinterpret_cast<uint32_t *>(region + 8u * V);
+  uint16_t *loc_g = reinterpret_cast<uint16_t *>(region + 12u * V);
+  // small tasks: the previous rebuild's survivors (both lists) are the prune's first filter
+  const uint32_t n_filt = small ? min(c.f_len[t], V) : 0u;
+  for (uint32_t i = tid; i < n_filt; i += B) filt[i] = min((uint32_t)loc_g[i], V - 1u);
   uint32_t F = 0, F0 = 0;                 // entries emitted so far; length of the first list
   const uint32_t n_lists = c.stateful ? 2u : 1u;
   for (uint32_t list = 0; list < n_lists; ++list) {
     __syncthreads();
-    if (tid == 0) { s_total = 0; s_inlist = 0; }
+    if (tid == 0) { s_total = 0; s_inlist = 0; s_ncand = 0; }
     __syncthreads();
     // 1. queue recursion and states (first pass), predicted latency, sort keys
     uint32_t mine = 0;
@@ -455,16 +472,22 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       uint32_t cost = 0, lat_key = 0, inv = 0;
       if (i < V) {
         const uint32_t slot = base + i;
-        uint32_t pred;
+        // every load before the first store: the arrays may alias as far as the compiler can
+        // tell, and each dependent round trip to memory costs about a microsecond here
+        const uint32_t acc = c.s_acc[slot];
+        uint32_t st = INFAAS_STATE_ACTIVE, load_lat = 0, pred;
+        cost = c.s_cost[slot];
+        if (c.stateful) { st = c.s_state[slot]; load_lat = c.s_load_lat[slot]; }
         if (list == 0) {
           const uint32_t lat = c.s_lat[slot];
           const uint32_t batch = c.s_batch[slot];
           uint32_t queued = c.s_queued[slot];
           if (advance) {
             const uint32_t id = c.s_id[slot];
+            const unsigned long long served = c.s_served[slot];
             const uint32_t cnt = c.count_by_id[id];
             c.count_by_id[id] = 0;
-            c.s_served[slot] += cnt;
+            c.s_served[slot] = served + cnt;
             unsigned long long arrived = (unsigned long long)queued + cnt;
             if (arrived > U32_MAX_) arrived = U32_MAX_;
             unsigned long long drain = (unsigned long long)window_us * batch / lat;
@@ -473,7 +496,6 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
             c.s_queued[slot] = queued;
             if (c.stateful) {
               // loaded by its first queries; at peak throughput while a backlog remains
-              uint32_t st = c.s_state[slot];
               if (st == INFAAS_STATE_INACTIVE && cnt > 0) st = INFAAS_STATE_ACTIVE;
               if (st == INFAAS_STATE_ACTIVE || st == INFAAS_STATE_OVERLOADED)
                 st = queued > 0 ? INFAAS_STATE_OVERLOADED : INFAAS_STATE_ACTIVE;
@@ -487,11 +509,11 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
           pred = c.s_pred[slot];
         }
         in = true;
-        cost = c.s_cost[slot]; lat_key = pred; inv = 10000u - c.s_acc[slot];
+        lat_key = pred; inv = 10000u - acc;
         if (c.stateful) {
-          in = c.s_state[slot] == (list == 0 ? INFAAS_STATE_ACTIVE : INFAAS_STATE_INACTIVE);
+          in = st == (list == 0 ? INFAAS_STATE_ACTIVE : INFAAS_STATE_INACTIVE);
           if (list == 1) {
-            const unsigned long long e = (unsigned long long)pred + c.s_load_lat[slot];
+            const unsigned long long e = (unsigned long long)pred + load_lat;
             cost = lat_key = e > U32_MAX_ ? U32_MAX_ : (uint32_t)e;
           }
         }
@@ -517,21 +539,39 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       // 3 (small tasks, before any sort).  q dominates p iff cost_q <= cost_p, pred_q <= pred_p,
       // acc_q >= acc_p and it differs in some attribute or has the smaller id -- which, given
       // the three inequalities, is the same as its key (cost, pred, 10000-acc, local index)
-      // being smaller.  G lanes share an entry's comparisons.
+      // being smaller.  Two rounds.  First every entry is tested against a filter set only,
+      // the survivors of the previous rebuild: whatever one of them dominates is gone, whatever
+      // set is used.  Then the entries that are left (every non-dominated entry is among them,
+      // and, dominance being transitive, each dominated one is dominated by one of those) are
+      // tested against each other.  The load moves little from window to window, so the second
+      // round sees few entries.  G lanes share an entry's comparisons in the first round.
       const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
       uint32_t dom = 0;
       if (p < V) {
         const uint4 a = attr[p];
         if (a.z == ~0u) dom = 1;                         // not in this list
         else
-          for (uint32_t q = sidx; q < V; q += G) {
-            const uint4 b = attr[q];                       // (cost, pred, 10000 - acc, local index)
-            if (b.x <= a.x && b.y <= a.y && b.z <= a.z)    // rare
+          for (uint32_t j = sidx; j < n_filt; j += G) {
+            const uint4 b = attr[filt[j]];                 // (cost, pred, 10000 - acc, local index)
+            if (b.x <= a.x && b.y <= a.y && b.z <= a.z)
               dom |= (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w) ? 1u : 0u;
           }
       }
       for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
-      if (p < V && sidx == 0) { keep[p] = !dom; my_kept = !dom; }
+      if (p < V && sidx == 0) {
+        keep[p] = !dom;
+        if (!dom) cand[atomicAdd(&s_ncand, 1u)] = (uint16_t)p;   // in any order
+      }
+      __syncthreads();
+      const uint32_t R = s_ncand;
+      for (uint32_t x = tid; x < R * R; x += B) {
+        const uint32_t ip = x / R, pp = cand[ip], qq = cand[x - ip * R];
+        const uint4 a = attr[pp], b = attr[qq];
+        if (b.x <= a.x && b.y <= a.y && b.z <= a.z && (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w))
+          keep[pp] = 0;                                    // several writers, one value
+      }
+      __syncthreads();
+      if (tid < V) my_kept = keep[tid];
     } else {
       // 2. bitonic sort of P keys, ascending in (cost, pred, 10000-acc, local index); what is
       // not in this list sorts behind it
@@ -583,6 +623,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       const uint32_t id = c.s_id[base + (v32 & 0xFFFFu)];
       keys_g[F + pos] = ((unsigned long long)acc << 32) | pred_p;
       ids_g[F + pos] = id;
+      loc_g[F + pos] = (uint16_t)(v32 & 0xFFFFu);
       if (list == 0 && pos < INDEX_MAX_F) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }   // first segment
     };
     uint32_t kept_so_far = 0;
@@ -618,6 +659,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     F += Fl;
   }
   bool indexed = F > 0;
+  bool counted = false;                       // has this CTA made its last allocation?
   // index the lists segment by segment (INDEX_MAX_F positions each; almost always one)
   if (indexed) {
     const uint32_t segs0 = (F0 + INDEX_MAX_F - 1u) / INDEX_MAX_F;
@@ -634,8 +676,10 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
         __syncthreads();
       }
       indexed = build_index(c, t, Fseg, S, sg ? x0 + sg - 1u : 0xFFFFFFFFu, sg + 1u < nseg ? x0 + sg + 1u : 0u);
+      counted = sg + 1u == nseg;
     }
   }
+  if (!counted && tid == 0) place_block(c, 0u, true);   // nothing (more) to place
   if (!indexed) {
     // no index: header and records that make every query of this task read "none"
     write_header(c, t, dummy_header(c.n_tasks));
@@ -651,29 +695,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     for (uint32_t j = tid; j < SLO_BUCKETS; j += B) rec[j] = 0u;
     if (tid < 16) reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid == 3 ? PENDING : 0u;
   }
-  if (tid == 0) {
-    c.f_len[t] = F;
-    atomicMax(&c.rebuild_ctr[2], F);
-    atomicAdd(&c.rebuild_ctr[3], F);
-    if (F > 0 && !indexed) atomicAdd(&c.rebuild_ctr[4], 1u);
-  }
-
-  // 5. the CTA that finishes last publishes the totals and resets the counters
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    uint32_t ticket = atomicAdd(&c.rebuild_ctr[0], 1u);
-    s_last = (ticket == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!s_last || tid != 0) return;
-  __threadfence();
-  volatile uint32_t *ctr = c.rebuild_ctr;
-  c.image_hdr[0] = image_var_offset(c.n_tasks) + ctr[1];
-  c.image_hdr[1] = ctr[2];
-  c.image_hdr[2] = ctr[3];
-  c.image_hdr[3] = ctr[4];
-  ctr[0] = 0; ctr[1] = 0; ctr[2] = 0; ctr[3] = 0; ctr[4] = 0;
+  if (tid == 0) c.f_len[t] = F;
 }
 
 }  // namespace
