@@ -212,9 +212,14 @@ __device__ __forceinline__ uint32_t group8_or(uint32_t v) {
 // One atomic per allocation places a block in the image and, on a CTA's last allocation
 // (`done`), counts the CTA as finished with the cursor.  The CTA that is counted last knows the
 // final image size: it publishes it for the kernels that follow and clears the counter for the
-// next rebuild.  Thread 0 only; returns the block's offset behind the fixed part of the image.
-__device__ __forceinline__ uint32_t place_block(const DeviceCatalog &c, uint32_t bytes, bool done) {
-  const unsigned long long old = atomicAdd(c.alloc_ctr, ((unsigned long long)(done ? 1u : 0u) << 32) | bytes);
+// next rebuild.  Thread 0 only, in two halves so that the atomic's round trip can overlap other
+// work: place_block_issue returns the counter's old value, place_block_finish (same arguments)
+// the block's offset behind the fixed part of the image.
+__device__ __forceinline__ unsigned long long place_block_issue(const DeviceCatalog &c, uint32_t bytes, bool done) {
+  return atomicAdd(c.alloc_ctr, ((unsigned long long)(done ? 1u : 0u) << 32) | bytes);
+}
+__device__ __forceinline__ uint32_t place_block_finish(const DeviceCatalog &c, unsigned long long old,
+                                                       uint32_t bytes, bool done) {
   if (done && (uint32_t)(old >> 32) == gridDim.x - 1u) {
     c.image_hdr[0] = image_var_offset(c.n_tasks) + (uint32_t)old + bytes;
     *c.alloc_ctr = 0ull;
@@ -279,6 +284,16 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   }
   __syncthreads();
   const uint32_t Ks = S.ks, Ka = S.ka, Fs = S.fs;
+  // block layout and its place in the image; the atomic that places it is in flight while the
+  // masks below are built
+  const uint32_t acc_lo = (S.Ad[0] / ACC_WORD_BITS) * ACC_WORD_BITS;
+  const uint32_t nbw = (S.Ad[Ka - 1] + 1u - acc_lo) / ACC_WORD_BITS + 1u;
+  const uint32_t width = Ka + 1u;
+  const BlockLayout BL = block_layout(F, Ks, Ka, nbw);
+  const SlowLayout SL = slow_layout(F, Ks, Ka);
+  const bool fits = nbw <= MAX_ACC_WORDS;
+  unsigned long long placed = 0;
+  if (tid == 0) placed = place_block_issue(c, fits ? BL.bytes : 0u, next == 0u);
   // SLO buckets: they cover the list's latencies up to the largest SLO asked for so far (as a
   // bit mask: every SLO seen is <= cap); larger latencies share bucket 255
   uint32_t cap = *c.slo_seen | SLO_CAP_FLOOR_US;
@@ -305,15 +320,8 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     (which ? S.Amask : S.Lmask)[rk][w] = m;
   }
 
-  // block layout and its place in the image
-  const uint32_t acc_lo = (S.Ad[0] / ACC_WORD_BITS) * ACC_WORD_BITS;
-  const uint32_t nbw = (S.Ad[Ka - 1] + 1u - acc_lo) / ACC_WORD_BITS + 1u;
-  const uint32_t width = Ka + 1u;
-  const BlockLayout BL = block_layout(F, Ks, Ka, nbw);
-  const SlowLayout SL = slow_layout(F, Ks, Ka);
   if (tid == 0) {
-    const bool fits = nbw <= MAX_ACC_WORDS;
-    uint32_t base = image_var_offset(c.n_tasks) + place_block(c, fits ? BL.bytes : 0u, next == 0u);
+    uint32_t base = image_var_offset(c.n_tasks) + place_block_finish(c, placed, fits ? BL.bytes : 0u, next == 0u);
     if (!fits || base + BL.bytes > c.image_capacity || base + BL.t2 >= IMAGE_T2_LIMIT) base = 0xFFFFFFFFu;
     S.base = base;
   }
@@ -442,12 +450,9 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint32_t P = 1;
   while (P < V) P <<= 1;
 
-  // small tasks have, behind the sort buffers, a second copy of the keys (survivors of the
-  // prune) and the attributes packed for the prune
+  // small tasks have, behind the sort buffers, the attributes packed for the prune
   const bool small = sort_n <= RANK_SORT_MAX;
-  unsigned long long *o64 = reinterpret_cast<unsigned long long *>(keep + sort_n + ((16u - ((13u * sort_n) & 15u)) & 15u));
-  uint32_t *o32 = reinterpret_cast<uint32_t *>(o64 + sort_n);
-  uint4 *attr = reinterpret_cast<uint4 *>((reinterpret_cast<uintptr_t>(o32 + sort_n) + 15u) & ~(uintptr_t)15u);
+  uint4 *attr = reinterpret_cast<uint4 *>((reinterpret_cast<uintptr_t>(keep + sort_n) + 15u) & ~(uintptr_t)15u);
 
   // A state-aware catalog has two lists per task: Active variants keyed (cost, pred, 10000-acc,
   // id), then Inactive ones keyed by their combined loading + inference latency, which takes
@@ -559,9 +564,14 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
           }
       }
       for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
-      if (p < V && sidx == 0) {
-        keep[p] = !dom;
-        if (!dom) cand[atomicAdd(&s_ncand, 1u)] = (uint16_t)p;   // in any order
+      {
+        const bool is_cand = p < V && sidx == 0 && !dom;
+        if (p < V && sidx == 0) keep[p] = !dom;
+        const unsigned m = __ballot_sync(0xFFFFFFFFu, is_cand);   // one append per warp, in any order
+        uint32_t at = 0;
+        if (m && (tid & 31u) == (uint32_t)__ffs(m) - 1u) at = atomicAdd(&s_ncand, (uint32_t)__popc(m));
+        at = __shfl_sync(0xFFFFFFFFu, at, m ? __ffs(m) - 1 : 0);
+        if (is_cand) cand[at + __popc(m & ((1u << (tid & 31u)) - 1u))] = (uint16_t)p;
       }
       __syncthreads();
       const uint32_t R = s_ncand;
@@ -627,35 +637,41 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       loc_g[F + pos] = (uint16_t)(v32 & 0xFFFFu);
       if (list == 0 && pos < INDEX_MAX_F) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }   // first segment
     };
-    uint32_t kept_so_far = 0;
-    for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
-      const uint32_t p = p0 + tid;
-      const bool kp = p < V && keep[p];
-      uint32_t total;
-      const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
-      if (kp) {
-        if (small) { o64[pos] = k64[p]; o32[pos] = k32[p]; }      // survivors, not yet in order
-        else emit(pos, k64[p], k32[p]);
+    if (!small) {
+      uint32_t kept_so_far = 0;
+      for (uint32_t p0 = 0; p0 < V; p0 += B) {      // uniform trip count
+        const uint32_t p = p0 + tid;
+        const bool kp = p < V && keep[p];
+        uint32_t total;
+        const uint32_t pos = kept_so_far + block_excl_scan_flag(kp, warp_sums, total);
+        if (kp) emit(pos, k64[p], k32[p]);
+        kept_so_far += total;
       }
-      kept_so_far += total;
-    }
-    __syncthreads();
-    if (small) {
-      // 2 (small tasks): the survivors' list positions by counting smaller keys
-      uint32_t PF = 1;
-      while (PF < Fl) PF <<= 1;
-      const uint32_t G = min(32u, B / PF), i = tid / G, sidx = tid % G;
+    } else {
+      // 2 (small tasks): the survivors' list positions by counting smaller keys among the
+      // second round's candidates, of which the survivors are most
+      const uint32_t R = s_ncand;
+      uint32_t PR = 1;
+      while (PR < R) PR <<= 1;
+      const uint32_t G = min(32u, B / PR), i = tid / G, sidx = tid % G;
       uint32_t rank = 0;
       unsigned long long a64 = 0;
       uint32_t a32 = 0;
-      if (i < Fl) {
-        a64 = o64[i]; a32 = o32[i];
-        for (uint32_t j = sidx; j < Fl; j += G) rank += key_less(o64[j], o32[j], a64, a32);
+      bool mine_kept = false;
+      if (i < R) {
+        const uint32_t pp = cand[i];
+        mine_kept = keep[pp];
+        a64 = k64[pp]; a32 = k32[pp];
+        if (mine_kept)
+          for (uint32_t j = sidx; j < R; j += G) {
+            const uint32_t qq = cand[j];
+            rank += keep[qq] && key_less(k64[qq], k32[qq], a64, a32);
+          }
       }
       for (uint32_t o = G >> 1; o; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
-      if (i < Fl && sidx == 0) emit(rank, a64, a32);
-      __syncthreads();
+      if (mine_kept && sidx == 0) emit(rank, a64, a32);
     }
+    __syncthreads();
     if (list == 0) F0 = Fl;
     F += Fl;
   }
@@ -680,7 +696,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       counted = sg + 1u == nseg;
     }
   }
-  if (!counted && tid == 0) place_block(c, 0u, true);   // nothing (more) to place
+  if (!counted && tid == 0) place_block_finish(c, place_block_issue(c, 0u, true), 0u, true);   // nothing (more) to place
   if (!indexed) {
     // no index: header and records that make every query of this task read "none"
     write_header(c, t, dummy_header(c.n_tasks));
@@ -739,8 +755,8 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream) {
   uint32_t P = 1;
   while (P < c.max_task_variants) P <<= 1;
-  // small tasks: room for a second copy of the keys (12 bytes per entry) and the packed attributes (16)
-  size_t smem = (size_t)P * 13 + (P <= RANK_SORT_MAX ? (size_t)P * 28 + 32 : 0);
+  // small tasks: room for the packed attributes (16 bytes per entry)
+  size_t smem = (size_t)P * 13 + (P <= RANK_SORT_MAX ? (size_t)P * 16 + 32 : 0);
   rebuild_kernel<<<c.n_tasks, REBUILD_THREADS, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
   return cudaGetLastError();
 }
