@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, from the ncu capture summarised in profiles/select_kernel_C3.md, per query (part of
 # the decisions is still in L2 when the kernel ends, hence below 12 B).  Set to None when the
 # kernel changes until the counters are taken again.
-NCU_TRAFFIC_BYTES_PER_QUERY = (134.56e6 + 27.22e6) / (1 << 24)
+NCU_TRAFFIC_BYTES_PER_QUERY = (134.54e6 + 26.94e6) / (1 << 24)
 
 
 def parse_args():
