@@ -35,6 +35,12 @@ FALLBACK_HBM_GBS = 6650.0
 # the decisions is still in L2 when the kernel ends, hence below 12 B).  Set to None when the
 # kernel changes until the counters are taken again.
 NCU_TRAFFIC_BYTES_PER_QUERY = (134.54e6 + 26.94e6) / (1 << 24)
+# From the same capture: warp-instructions executed and shared-memory wavefronts (one per
+# clock and SM at most) per query, for the two on-chip limits the kernel sits closer to than
+# to HBM.  Same rule as above when the kernel changes.
+NCU_WARP_INSTR_PER_QUERY = 41.39e6 / (1 << 24)
+NCU_SMEM_WAVEFRONTS_PER_QUERY = 10.30e6 / (1 << 24)
+SM_COUNT, ISSUE_PER_SM_CLK = 148, 4
 
 
 def parse_args():
@@ -50,6 +56,15 @@ def parse_args():
     ap.add_argument("--split-update", action="store_true",
                     help="with one rank too, update through tally / count exchange / advance (the N > 1 path)")
     return ap.parse_args()
+
+
+def on_chip_limits(n: int, sel_ms: float, sm_mhz):
+    if not sm_mhz or NCU_WARP_INSTR_PER_QUERY is None:
+        return None
+    clk = SM_COUNT * sm_mhz * 1e6 * sel_ms * 1e-3              # SM-clocks available to the launch
+    return {"issue_slot_frac": NCU_WARP_INSTR_PER_QUERY * n / (ISSUE_PER_SM_CLK * clk),
+            "smem_wavefront_frac": NCU_SMEM_WAVEFRONTS_PER_QUERY * n / clk,
+            "how": "ncu instruction and wavefront counts per query x queries / (SMs x clock x time)"}
 
 
 def make_workload(name: str, queries: int):
@@ -304,6 +319,9 @@ def run_ours(args):
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "traffic": None if NCU_TRAFFIC_BYTES_PER_QUERY is None
                      else NCU_TRAFFIC_BYTES_PER_QUERY * n},
+        # the same launch against the SM's own limits at the clock sampled during the run:
+        # issue slots (4 warp-instructions per SM and clock) and shared-memory wavefronts (1)
+        "on_chip_limits": on_chip_limits(n, sel_avg_ms, clocks.summary().get("sm_mhz")),
         "clocks": clocks.summary(),
         "decisions": {"feasible": int(((dec_host >> 31) == 0).sum()),
                       "no_feasible": int((((dec_host >> 31) == 1) & (dec_host != 0xFFFFFFFF)).sum()),
