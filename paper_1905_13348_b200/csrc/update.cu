@@ -438,8 +438,9 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
   unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
-  __shared__ uint32_t s_total, s_inlist, s_ncand;
-  __shared__ uint16_t filt[RANK_SORT_MAX], cand[RANK_SORT_MAX];   // small tasks: filter set, candidates
+  __shared__ uint32_t s_total, s_inlist, s_ncand, s_nnew;
+  __shared__ uint16_t filt[RANK_SORT_MAX], cand[RANK_SORT_MAX], newc[RANK_SORT_MAX];   // small tasks: filter set,
+  __shared__ unsigned char in_filt[RANK_SORT_MAX];                // candidates, those of them not in the filter set
   __shared__ IndexScratch S;
 
   const uint32_t t = blockIdx.x, tid = threadIdx.x, B = blockDim.x;
@@ -463,12 +464,20 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   uint16_t *loc_g = reinterpret_cast<uint16_t *>(region + 12u * V);
   // small tasks: the previous rebuild's survivors (both lists) are the prune's first filter
   const uint32_t n_filt = small ? min(c.f_len[t], V) : 0u;
-  for (uint32_t i = tid; i < n_filt; i += B) filt[i] = min((uint32_t)loc_g[i], V - 1u);
+  if (small) {
+    for (uint32_t i = tid; i < V; i += B) in_filt[i] = 0;
+    __syncthreads();
+    for (uint32_t i = tid; i < n_filt; i += B) {
+      const uint32_t f = min((uint32_t)loc_g[i], V - 1u);
+      filt[i] = (uint16_t)f;
+      in_filt[f] = 1;
+    }
+  }
   uint32_t F = 0, F0 = 0;                 // entries emitted so far; length of the first list
   const uint32_t n_lists = c.stateful ? 2u : 1u;
   for (uint32_t list = 0; list < n_lists; ++list) {
     __syncthreads();
-    if (tid == 0) { s_total = 0; s_inlist = 0; s_ncand = 0; }
+    if (tid == 0) { s_total = 0; s_inlist = 0; s_ncand = 0; s_nnew = 0; }
     __syncthreads();
     // 1. queue recursion and states (first pass), predicted latency, sort keys
     uint32_t mine = 0;
@@ -547,10 +556,12 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       // the three inequalities, is the same as its key (cost, pred, 10000-acc, local index)
       // being smaller.  Two rounds.  First every entry is tested against a filter set only,
       // the survivors of the previous rebuild: whatever one of them dominates is gone, whatever
-      // set is used.  Then the entries that are left (every non-dominated entry is among them,
-      // and, dominance being transitive, each dominated one is dominated by one of those) are
-      // tested against each other.  The load moves little from window to window, so the second
-      // round sees few entries.  G lanes share an entry's comparisons in the first round.
+      // set is used.  Every non-dominated entry is among the entries that are left, and,
+      // dominance being transitive, each dominated one is dominated by one of those; against the
+      // ones inside the filter set it has been tested already, so the second round tests the
+      // entries that are left against those of them outside the filter set.  The load moves
+      // little from window to window, so these are few.  G lanes share an entry's comparisons
+      // in the first round.
       const uint32_t G = min(32u, B / P), p = tid / G, sidx = tid % G;
       uint32_t dom = 0;
       if (p < V) {
@@ -572,11 +583,18 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
         if (m && (tid & 31u) == (uint32_t)__ffs(m) - 1u) at = atomicAdd(&s_ncand, (uint32_t)__popc(m));
         at = __shfl_sync(0xFFFFFFFFu, at, m ? __ffs(m) - 1 : 0);
         if (is_cand) cand[at + __popc(m & ((1u << (tid & 31u)) - 1u))] = (uint16_t)p;
+        // candidates outside the filter set: the only ones the first round has not tested the others against
+        const bool is_new = is_cand && !in_filt[p];
+        const unsigned mn = __ballot_sync(0xFFFFFFFFu, is_new);
+        uint32_t an = 0;
+        if (mn && (tid & 31u) == (uint32_t)__ffs(mn) - 1u) an = atomicAdd(&s_nnew, (uint32_t)__popc(mn));
+        an = __shfl_sync(0xFFFFFFFFu, an, mn ? __ffs(mn) - 1 : 0);
+        if (is_new) newc[an + __popc(mn & ((1u << (tid & 31u)) - 1u))] = (uint16_t)p;
       }
       __syncthreads();
-      const uint32_t R = s_ncand;
-      for (uint32_t x = tid; x < R * R; x += B) {
-        const uint32_t ip = x / R, pp = cand[ip], qq = cand[x - ip * R];
+      const uint32_t R = s_ncand, Nn = s_nnew;
+      for (uint32_t x = tid; x < R * Nn; x += B) {
+        const uint32_t ip = x / Nn, pp = cand[ip], qq = newc[x - ip * Nn];
         const uint4 a = attr[pp], b = attr[qq];
         if (b.x <= a.x && b.y <= a.y && b.z <= a.z && (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w))
           keep[pp] = 0;                                    // several writers, one value
