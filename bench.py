@@ -334,7 +334,10 @@ def run_ours(args):
         out["select_only"] = {"value": world * n / (sel_avg_ms * 1e-3), "unit": UNIT, "ms": sel_avg_ms}
         out["e2e"] = e2e_leg(P, cat, w, dev, update, max(3, min(10, args.steps)), world, dist)
         if w.window and world == 1:
-            out["windowed"] = windowed_leg(P, cat, w, inputs[0], d_dec, world)
+            # from the workload's own initial state, whatever the steps above left behind
+            cat_w = P.infaas_catalog_load(w.rows, w.n_tasks, local)
+            out["windowed"] = windowed_leg(P, cat_w, w, inputs[0], d_dec, world)
+            cat_w.free()
             out["stateful"] = stateful_leg(P, w, inputs, d_dec, local, peak)
             out["autoscale"] = autoscale_leg(P, w, inputs[0], d_dec, local)
             out["workers"] = workers_leg(P, w, cat, d_dec, peak)
@@ -431,7 +434,9 @@ def e2e_leg(P, cat, w, dev, update, steps, world, dist):
 def windowed_leg(P, cat, w, inp, d_dec, world):
     """The workload as a stream of windows: select one window, update the load, repeat.
     All windows are captured once into a CUDA graph (the calls only launch kernels), so the
-    timing shows the device-side dependency chain and not the Python call overhead."""
+    timing shows the device-side dependency chain and not the Python call overhead.  The
+    catalog keeps its load from one pass over the windows to the next: the timed passes are
+    the fourth to the eighth, when the queues have settled."""
     import torch
     t, s, a = inp
     W_ = w.window
@@ -452,6 +457,7 @@ def windowed_leg(P, cat, w, inp, d_dec, world):
         run(side)
         side.synchronize()
         eager_ms = 1e3 * (time.perf_counter() - t0)
+        P.infaas_catalog_get_state(cat, stream=side)   # lets the library re-plan its shared memory for the lists as they are now
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
             run(side)
@@ -465,7 +471,9 @@ def windowed_leg(P, cat, w, inp, d_dec, world):
         e1.record(side)
         side.synchronize()
     ms = e0.elapsed_time(e1) / reps
+    info = P.infaas_catalog_get_info(cat, stream=side)
     return {"value": world * nwin * W_ / (ms * 1e-3), "unit": UNIT, "windows": nwin,
+            "windows_before_timing": 3 * nwin, "lists_after": {k: info[k] for k in ("image_bytes", "longest_list", "list_entries")},
             "window_queries": W_, "us_per_window": 1e3 * ms / nwin, "gpu_launches_per_window": 3,
             "how": "CUDA graph of all windows", "us_per_window_python_calls": 1e3 * eager_ms / nwin}
 

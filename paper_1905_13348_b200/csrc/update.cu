@@ -144,7 +144,13 @@ tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_
 // ------------------------------------------------------------------------------------
 __device__ __forceinline__ bool key_less(unsigned long long a64, uint32_t a32,
                                          unsigned long long b64, uint32_t b32) {
-  return a64 < b64 || (a64 == b64 && a32 < b32);
+  return (a64 < b64) | ((a64 == b64) & (a32 < b32));
+}
+// Packed attributes (cost, pred, 10000 - acc, local index): does b dominate a?  Not worse in
+// any of the three, and different in one of them or with the smaller index.  Branch-free.
+__device__ __forceinline__ uint32_t dominates(const uint4 b, const uint4 a) {
+  return (uint32_t)((b.x <= a.x) & (b.y <= a.y) & (b.z <= a.z) &
+                    ((b.x != a.x) | (b.y != a.y) | (b.z != a.z) | (b.w < a.w)));
 }
 
 // Exclusive scan of one flag per thread over the CTA; returns this thread's offset and the
@@ -434,7 +440,11 @@ constexpr uint32_t RANK_SORT_MAX = 512;   // tasks up to this size are sorted by
 __global__ void __launch_bounds__(REBUILD_THREADS)
 rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned long long *k64 = reinterpret_cast<unsigned long long *>(smem_raw);   // cost<<32 | pred
+  // small tasks have, in front of the sort buffers, the attributes packed for the prune (kept a
+  // plain offset from the shared array so that the loads stay shared-memory loads)
+  const bool small = sort_n <= RANK_SORT_MAX;
+  uint4 *attr = reinterpret_cast<uint4 *>(smem_raw);
+  unsigned long long *k64 = reinterpret_cast<unsigned long long *>(smem_raw + (small ? 16u * sort_n : 0u));   // cost<<32 | pred
   uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
   unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
@@ -450,10 +460,6 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   // sort size for this task: the power of two that holds it (tasks differ in size)
   uint32_t P = 1;
   while (P < V) P <<= 1;
-
-  // small tasks have, behind the sort buffers, the attributes packed for the prune
-  const bool small = sort_n <= RANK_SORT_MAX;
-  uint4 *attr = reinterpret_cast<uint4 *>((reinterpret_cast<uintptr_t>(keep + sort_n) + 15u) & ~(uintptr_t)15u);
 
   // A state-aware catalog has two lists per task: Active variants keyed (cost, pred, 10000-acc,
   // id), then Inactive ones keyed by their combined loading + inference latency, which takes
@@ -567,12 +573,13 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       if (p < V) {
         const uint4 a = attr[p];
         if (a.z == ~0u) dom = 1;                         // not in this list
-        else
-          for (uint32_t j = sidx; j < n_filt; j += G) {
+        else {
+#pragma unroll 4
+          for (uint32_t j = sidx; j < n_filt; j += G) {    // no branch: the loads of several trips overlap
             const uint4 b = attr[filt[j]];                 // (cost, pred, 10000 - acc, local index)
-            if (b.x <= a.x && b.y <= a.y && b.z <= a.z)
-              dom |= (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w) ? 1u : 0u;
+            dom |= dominates(b, a);
           }
+        }
       }
       for (uint32_t o = G >> 1; o; o >>= 1) dom |= __shfl_xor_sync(0xFFFFFFFFu, dom, o);   // lane-aligned groups
       {
@@ -595,9 +602,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       const uint32_t R = s_ncand, Nn = s_nnew;
       for (uint32_t x = tid; x < R * Nn; x += B) {
         const uint32_t ip = x / Nn, pp = cand[ip], qq = newc[x - ip * Nn];
-        const uint4 a = attr[pp], b = attr[qq];
-        if (b.x <= a.x && b.y <= a.y && b.z <= a.z && (b.x != a.x || b.y != a.y || b.z != a.z || b.w < a.w))
-          keep[pp] = 0;                                    // several writers, one value
+        if (dominates(attr[qq], attr[pp])) keep[pp] = 0;   // several writers, one value
       }
       __syncthreads();
       if (tid < V) my_kept = keep[tid];
@@ -680,11 +685,13 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
         const uint32_t pp = cand[i];
         mine_kept = keep[pp];
         a64 = k64[pp]; a32 = k32[pp];
-        if (mine_kept)
+        if (mine_kept) {
+#pragma unroll 4
           for (uint32_t j = sidx; j < R; j += G) {
             const uint32_t qq = cand[j];
-            rank += keep[qq] && key_less(k64[qq], k32[qq], a64, a32);
+            rank += (uint32_t)keep[qq] & (uint32_t)key_less(k64[qq], k32[qq], a64, a32);
           }
+        }
       }
       for (uint32_t o = G >> 1; o; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
       if (mine_kept && sidx == 0) emit(rank, a64, a32);
