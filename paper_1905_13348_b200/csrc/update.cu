@@ -346,15 +346,21 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
 
   // T2: cell (r, k) = first position whose latency rank is < r and accuracy rank >= k
   unsigned char *T2 = blk + BL.t2;
-  share(0, B / 2, (Ks + 2u) * width, [&](uint32_t cell) {
-    const uint32_t r = cell / width, k = cell - r * width;
-    uint32_t pos = F;
-    if (r >= 1 && r <= Ks)
-      for (uint32_t w = 0; w < nw; ++w) {
-        const unsigned long long m = S.Lmask[r][w] & S.Amask[k][w];
-        if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
-      }
-    T2[cell] = (unsigned char)pos;
+  // four consecutive cells per step, stored as one word (the table is padded to a multiple of 4)
+  share(0, B / 2, ((Ks + 2u) * width + 3u) >> 2, [&](uint32_t q) {
+    uint32_t r = (q << 2) / width, k = (q << 2) - r * width, word = 0;
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) {
+      uint32_t pos = F;
+      if (r >= 1 && r <= Ks)
+        for (uint32_t w = 0; w < nw; ++w) {
+          const unsigned long long m = S.Lmask[r][w] & S.Amask[k][w];
+          if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
+        }
+      word |= pos << (8u * u);
+      if (++k == width) { k = 0; ++r; }
+    }
+    reinterpret_cast<uint32_t *>(T2)[q] = word;            // cells past the last row hold F
   });
 
   // SLO records (see common.cuh)
