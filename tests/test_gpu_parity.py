@@ -383,3 +383,32 @@ def test_random_catalog_shapes(seed):
     q_acc = np.where(rng.random(n) < 0.9, rng.integers(0, 10001, n), rng.choice(np.array([0, 10001, 65535]), n)).astype(np.uint16)
     w = W.Workload("shapes", T, rows, q_task, q_slo, q_acc, 20011, 50_000, "random shapes")
     run_both(w)
+
+
+def test_image_somewhat_larger_than_shared_memory():
+    # windows short enough for the queues to be noisy: the lists grow until the lookup image no
+    # longer fits in shared memory; the kernel then reads it from global memory, first with the
+    # shared memory still reserved, then (after the next look at the state) without
+    import paper_1905_13348_b200 as P
+    win, n_win = 8192, 36
+    w = W.make("C3", n_queries=n_win * win, window=win)
+    w.window_us = 5000
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    reserved = released = 0
+    try:
+        for k in range(n_win):
+            s = slice(k * win, (k + 1) * win)
+            want = o.select(w.task[s], w.slo_us[s], w.min_acc_bp[s], 8)
+            d_dec = gpu_select(cat, w.task[s], w.slo_us[s], w.min_acc_bp[s])
+            assert np.array_equal(_to_host_u32(d_dec), want), k
+            info = P.infaas_catalog_get_info(cat)
+            reserved += info["image_smem"] > 0 and info["image_bytes"] > info["image_smem"]
+            released += info["image_smem"] == 0
+            P.infaas_load_update(cat, d_dec, w.window_us)
+            o.load_update(want, w.window_us)
+            if k % 4 == 3:
+                assert_state_equal(cat, o)        # also lets the library re-plan its shared memory
+        assert released >= 10, (reserved, released)
+    finally:
+        cat.free()
