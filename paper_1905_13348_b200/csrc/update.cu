@@ -187,8 +187,65 @@ struct IndexScratch {          // shared memory used while building one task's i
   uint16_t acc[256], Ad[256];
   unsigned char idxP[256], idxA[256], firstP[256], firstA[256], bucket[256], on_stair[256];
   unsigned long long Lmask[256][4], Amask[256][4];   // positions by latency rank < r / accuracy rank >= k
+  // per latency rank: the most accurate entry (acc << 16 | 0xFFFF - position, 0 = none) and
+  // 1 + position of its stair entry (0 = none); per accuracy rank: the fastest entry
+  // (pred << 32 | position, ~0 = none); then their running maximum / minimum / count
+  uint32_t rankA[256];
+  unsigned long long rankB[256];
+  uint16_t stair_at[256];
+  uint32_t bestA[257];
+  unsigned long long bestB[257];
+  unsigned char ord_start[257];
   uint32_t ks, ka, base, fs;
 };
+
+// Scans over at most 257 per-rank values by one warp, 32 at a time with a carry.
+// out[r] = max of in[0 .. r-1] (0 for r = 0), r = 0 .. n.
+__device__ __forceinline__ void warp_prefix_max(const uint32_t *in, uint32_t *out, uint32_t n) {
+  const uint32_t lane = threadIdx.x & 31u;
+  uint32_t carry = 0;
+  for (uint32_t c0 = 0; c0 <= n; c0 += 32) {
+    const uint32_t i = c0 + lane;
+    uint32_t x = i < n ? in[i] : 0u;
+#pragma unroll
+    for (uint32_t o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+      if (lane >= o) x = max(x, y);
+    }
+    uint32_t before = __shfl_up_sync(0xFFFFFFFFu, x, 1);
+    before = max(lane ? before : 0u, carry);
+    if (i <= n) out[i] = before;
+    carry = max(carry, __shfl_sync(0xFFFFFFFFu, x, 31));
+  }
+}
+// out[k] = min of in[k .. n-1] (~0 for k = n), k = 0 .. n.
+__device__ __forceinline__ void warp_suffix_min(const unsigned long long *in, unsigned long long *out, uint32_t n) {
+  const uint32_t lane = threadIdx.x & 31u;
+  unsigned long long carry = ~0ull;
+  if (lane == 0) out[n] = ~0ull;
+  for (uint32_t c0 = 0; c0 < n; c0 += 32) {              // from the top down
+    const uint32_t q = c0 + lane;                          // q-th element from the top
+    unsigned long long x = q < n ? in[n - 1u - q] : ~0ull;
+#pragma unroll
+    for (uint32_t o = 1; o < 32; o <<= 1) {
+      const unsigned long long y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+      if (lane >= o) x = min(x, y);
+    }
+    if (q < n) out[n - 1u - q] = min(x, carry);
+    carry = min(carry, __shfl_sync(0xFFFFFFFFu, x, 31));
+  }
+}
+// out[r] = number of non-zero in[0 .. r-1], r = 0 .. n.
+__device__ __forceinline__ void warp_prefix_count(const uint16_t *in, unsigned char *out, uint32_t n) {
+  const uint32_t lane = threadIdx.x & 31u;
+  uint32_t carry = 0;
+  for (uint32_t c0 = 0; c0 <= n; c0 += 32) {
+    const uint32_t i = c0 + lane;
+    const unsigned m = __ballot_sync(0xFFFFFFFFu, i < n && in[i] != 0);
+    if (i <= n) out[i] = (unsigned char)(carry + __popc(m & ((1u << lane) - 1u)));
+    carry += __popc(m);
+  }
+}
 
 // Header of a task without index (also entry n_tasks): every query reads "none".
 __device__ __forceinline__ uint4 dummy_header(uint32_t n_tasks) {
@@ -266,6 +323,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     if (p < F && sub == 0) { S.firstP[p] = !(dup & 1u); S.firstA[p] = !(dup & 2u); S.on_stair[p] = !(dup & 4u); }
   }
   if (tid == 0) { S.ks = 0; S.ka = 0; S.fs = 0; }
+  if (tid < 256) { S.rankA[tid] = 0u; S.rankB[tid] = ~0ull; S.stair_at[tid] = 0; }
   __syncthreads();
   // ... and their ranks
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {
@@ -285,11 +343,19 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
       S.Ad[ra] = S.acc[p];
       atomicMax(&S.ks, rp + 1);
       atomicMax(&S.ka, ra + 1);
-      if (S.on_stair[p]) atomicAdd(&S.fs, 1u);
+      if (S.on_stair[p]) { atomicAdd(&S.fs, 1u); S.stair_at[rp] = (uint16_t)(p + 1u); }   // one per latency
+      atomicMax(&S.rankA[rp], ((uint32_t)S.acc[p] << 16) | (0xFFFFu - p));       // most accurate, first position
+      atomicMin(&S.rankB[ra], ((unsigned long long)S.pred[p] << 32) | p);        // fastest, first position
     }
   }
   __syncthreads();
   const uint32_t Ks = S.ks, Ka = S.ka, Fs = S.fs;
+  // what the nearest-miss search reads, as running aggregates over the ranks (three warps, while
+  // the others start on the masks): bestA[r] over latency ranks < r, bestB[k] over accuracy ranks
+  // >= k, ord_start[r] = stair entries with latency rank < r
+  if ((tid >> 5) == 0) warp_prefix_max(S.rankA, S.bestA, Ks);
+  if ((tid >> 5) == 1) warp_suffix_min(S.rankB, S.bestB, Ka);
+  if ((tid >> 5) == 2) warp_prefix_count(S.stair_at, S.ord_start, Ks);
   // block layout and its place in the image; the atomic that places it is in flight while the
   // masks below are built
   const uint32_t acc_lo = (S.Ad[0] / ACC_WORD_BITS) * ACC_WORD_BITS;
@@ -396,36 +462,24 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     bitmap[w] = (prefix << 24) | bits;
   });
 
-  // what the nearest-miss search reads
+  // what the nearest-miss search reads (aggregated above): position 0xFF stands for "none"
   uint32_t *bestA = reinterpret_cast<uint32_t *>(slow + SL.bestA);
   share(7 * B / 8, B / 16, Ks + 1u, [&](uint32_t r) {
-    uint32_t best = 0xFFu, best_acc = 0, cnt = 0;               // highest accuracy among ranks < r
-    for (uint32_t p = 0; p < F; ++p) {
-      if (S.idxP[p] < r) {
-        cnt += S.on_stair[p];
-        if (best == 0xFFu || S.acc[p] > best_acc) { best = p; best_acc = S.acc[p]; }
-      }
-    }
-    bestA[r] = best_acc | (best << 16);
-    slow[SL.ordStart + r] = (unsigned char)cnt;
+    const uint32_t v = S.bestA[r];                               // highest accuracy among ranks < r
+    bestA[r] = v ? (v >> 16) | ((0xFFFFu - (v & 0xFFFFu)) << 16) : 0xFFu << 16;
+    slow[SL.ordStart + r] = S.ord_start[r];
   });
   uint2 *bestB = reinterpret_cast<uint2 *>(slow + SL.bestB);
   share(15 * B / 16, B / 16, Ka + 1u, [&](uint32_t k) {
-    uint32_t best = 0xFFu, best_pred = 0;                        // lowest latency among accuracy ranks >= k
-    for (uint32_t p = 0; p < F; ++p) {
-      if (S.idxA[p] >= k && (best == 0xFFu || S.pred[p] < best_pred)) { best = p; best_pred = S.pred[p]; }
-    }
-    bestB[k] = make_uint2(best_pred, best);
+    const unsigned long long v = S.bestB[k];                     // lowest latency among accuracy ranks >= k
+    bestB[k] = v == ~0ull ? make_uint2(0u, 0xFFu) : make_uint2((uint32_t)(v >> 32), (uint32_t)v);
   });
   // small copies, after the short loops above
   uint32_t *ids_end = reinterpret_cast<uint32_t *>(blk + BL.t2);   // ids, reversed; slot F holds PENDING
   share(3 * B / 4, B / 8, F + 1u, [&](uint32_t p) { ids_end[-1 - (int)p] = p < F ? S.ids[p] : PENDING; });
   uint2 *walk = reinterpret_cast<uint2 *>(slow + SL.walk);      // the stair entries, ascending latency
-  share(7 * B / 8, B / 16, F, [&](uint32_t p) {
-    if (!S.on_stair[p]) return;
-    uint32_t o = 0;                                             // stair entries have distinct latencies
-    for (uint32_t q = 0; q < F; ++q) o += S.on_stair[q] && S.pred[q] < S.pred[p];
-    walk[o] = make_uint2(S.pred[p], (uint32_t)S.acc[p] | (p << 16));
+  share(7 * B / 8, B / 16, F, [&](uint32_t p) {                // stair entries have distinct latencies
+    if (S.on_stair[p]) walk[S.ord_start[S.idxP[p]]] = make_uint2(S.pred[p], (uint32_t)S.acc[p] | (p << 16));
   });
   uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
   share(15 * B / 16, B / 16, Ks, [&](uint32_t i) { Pd_g[i] = S.Pd[i]; });
