@@ -185,7 +185,9 @@ constexpr uint32_t BITS_OF_2_POW_32 = 0x4F800000u;
 struct IndexScratch {          // shared memory used while building one task's index
   uint32_t pred[256], Pd[256], ids[256];
   uint16_t acc[256], Ad[256];
-  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], bucket[256], on_stair[256];
+  unsigned char idxP[256], idxA[256], firstP[256], firstA[256], on_stair[256];
+  uint32_t bcnt[256], bthr[256];    // per SLO bucket: distinct latencies inside it, one of them
+  uint32_t wbits[256];              // per bitmap word: the accuracies present
   unsigned long long Lmask[256][4], Amask[256][4];   // positions by latency rank < r / accuracy rank >= k
   // per latency rank: the most accurate entry (acc << 16 | 0xFFFF - position, 0 = none) and
   // 1 + position of its stair entry (0 = none); per accuracy rank: the fastest entry
@@ -323,7 +325,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     if (p < F && sub == 0) { S.firstP[p] = !(dup & 1u); S.firstA[p] = !(dup & 2u); S.on_stair[p] = !(dup & 4u); }
   }
   if (tid == 0) { S.ks = 0; S.ka = 0; S.fs = 0; }
-  if (tid < 256) { S.rankA[tid] = 0u; S.rankB[tid] = ~0ull; S.stair_at[tid] = 0; }
+  if (tid < 256) { S.rankA[tid] = 0u; S.rankB[tid] = ~0ull; S.stair_at[tid] = 0; S.bcnt[tid] = 0u; S.wbits[tid] = 0u; }
   __syncthreads();
   // ... and their ranks
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {
@@ -375,8 +377,15 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   uint32_t sh = 0;
   while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
   const uint32_t bmin = clo >> sh, Sh = 16u + sh;
-  for (uint32_t i = tid; i < Ks; i += B)
-    S.bucket[i] = (unsigned char)(min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1));
+  for (uint32_t i = tid; i < Ks; i += B) {
+    const uint32_t b = min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1);
+    atomicAdd(&S.bcnt[b], 1u);
+    S.bthr[b] = S.Pd[i];                                 // read only where it is the bucket's only one
+  }
+  for (uint32_t i = tid; i < Ka; i += B) {
+    const uint32_t x = S.Ad[i] - acc_lo, xw = x / ACC_WORD_BITS;
+    atomicOr(&S.wbits[xw], 1u << (x - xw * ACC_WORD_BITS));
+  }
   // position masks: Lmask[r] = positions whose latency rank is < r, Amask[k] = positions whose
   // accuracy rank is >= k (64 positions per word); T2[r][k] is the first bit of their intersection
   const uint32_t nw = (F + 63u) >> 6;
@@ -431,13 +440,21 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
 
   // SLO records (see common.cuh)
   uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
-  share(B / 2, B / 4, first ? SLO_BUCKETS : 0u, [&](uint32_t j) {
-    uint32_t lb = 0, cnt = 0, thr = 0;
-    for (uint32_t i = 0; i < Ks; ++i) {
-      const uint32_t b = S.bucket[i];
-      lb += b < j;
-      if (b == j) { ++cnt; thr = S.Pd[i]; }
+  // one bucket per thread of warps 16-23; lb = latencies in lower buckets: the lower warps'
+  // buckets summed by the lanes, then a scan inside the warp
+  if (first && tid >= B / 2 && tid < B / 2 + SLO_BUCKETS) {
+    const uint32_t j = tid - B / 2, lane = tid & 31u;
+    uint32_t below = 0;
+    for (uint32_t i = lane; i < (j & ~31u); i += 32) below += S.bcnt[i];
+    below = __reduce_add_sync(0xFFFFFFFFu, below);
+    const uint32_t cnt = S.bcnt[j], thr = S.bthr[j];
+    uint32_t incl = cnt;
+#pragma unroll
+    for (uint32_t o = 1; o < 32; o <<= 1) {
+      const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += y;
     }
+    const uint32_t lb = below + incl - cnt;
     const uint32_t lo = j ? float_bits_floor((bmin + j) << Sh) : 0u;
     const uint32_t next = (bmin + j + 1u) << Sh;
     const uint32_t hi = (j == SLO_BUCKETS - 1 || next >= BITS_OF_2_POW_32) ? 0xFFFFFFFFu : float_bits_floor(next) - 1u;
@@ -448,19 +465,27 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
       r = thr <= lo ? (lb + 1u) << 24 : (lb << 24) | (0x00FFFFFFu - ((thr - 1u) & 0x00FFFFFFu));
     }
     rec[j] = r;
-  });
+  }
 
-  // accuracy bitmap with running popcounts
+  // accuracy bitmap with running popcounts: warps 24-27, 128 words a round, same scheme
   uint32_t *bitmap = reinterpret_cast<uint32_t *>(blk + BL.bitmap);
-  share(3 * B / 4, B / 8, nbw, [&](uint32_t w) {
-    uint32_t bits = 0, prefix = 0;
-    for (uint32_t i = 0; i < Ka; ++i) {
-      const uint32_t x = S.Ad[i] - acc_lo, xw = x / ACC_WORD_BITS;
-      prefix += xw < w;
-      if (xw == w) bits |= 1u << (x - xw * ACC_WORD_BITS);
+  if (tid >= 3 * B / 4 && tid < 3 * B / 4 + 128u) {
+    const uint32_t lane = tid & 31u;
+    for (uint32_t w0 = 0; w0 < nbw; w0 += 128u) {              // uniform over the four warps
+      const uint32_t w = w0 + (tid - 3 * B / 4);
+      uint32_t below = 0;
+      for (uint32_t i = lane; i < (w & ~31u); i += 32) below += __popc(S.wbits[i]);
+      below = __reduce_add_sync(0xFFFFFFFFu, below);
+      const uint32_t bits = w < nbw ? S.wbits[w] : 0u, pc = __popc(bits);
+      uint32_t incl = pc;
+#pragma unroll
+      for (uint32_t o = 1; o < 32; o <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += y;
+      }
+      if (w < nbw) bitmap[w] = ((below + incl - pc) << 24) | bits;
     }
-    bitmap[w] = (prefix << 24) | bits;
-  });
+  }
 
   // what the nearest-miss search reads (aggregated above): position 0xFF stands for "none"
   uint32_t *bestA = reinterpret_cast<uint32_t *>(slow + SL.bestA);
@@ -495,6 +520,9 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
 }
 
 constexpr uint32_t REBUILD_THREADS = 1024;
+// build_index gives fixed warps fixed tables: warps 16-23 one SLO bucket per thread, warps 24-27
+// the bitmap words
+static_assert(REBUILD_THREADS == 1024 && SLO_BUCKETS == 256, "thread ranges of build_index");
 constexpr uint32_t RANK_SORT_MAX = 512;   // tasks up to this size are sorted by counting smaller keys
 
 __global__ void __launch_bounds__(REBUILD_THREADS)
