@@ -18,7 +18,8 @@ namespace infaas {
 // the order above, then the Inactive ones with pred_lat + loading latency (saturating) in
 // place of both cost and pred_lat; each list is pruned on its own, variants in other states
 // are in neither.  "First feasible position, else the smallest distance at the lowest
-// position" over the two lists in this order is the state-aware answer.
+// position" over the two lists in this order is the state-aware answer, and that is all the
+// index below knows about order, so the two lists are indexed as one.
 //
 // A list is cut into segments of at most INDEX_MAX_F consecutive positions (almost always
 // one).  The selection kernel's fast path looks at the first segment only; if that holds

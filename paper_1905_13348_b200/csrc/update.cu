@@ -311,14 +311,15 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {            // uniform trip count
     const uint32_t p = p0 + (tid >> 3);
     // bit 0: an earlier entry has this latency; bit 1: this accuracy; bit 2: some entry is at
-    // least as fast and at least as accurate, and better in one of the two
+    // least as fast and at least as accurate, and better in one of the two or, being equal in
+    // both (an Active and an Inactive entry can be), earlier
     uint32_t dup = 0;
     if (p < F) {
       const uint32_t pp = S.pred[p], pa = S.acc[p];
       for (uint32_t q = sub; q < F; q += 8) {
         const uint32_t qp = S.pred[q], qa = S.acc[q];
         if (q < p) dup |= (qp == pp ? 1u : 0u) | (qa == pa ? 2u : 0u);
-        dup |= (qp <= pp && qa >= pa && (qp < pp || qa > pa)) ? 4u : 0u;
+        dup |= (qp <= pp && qa >= pa && (qp < pp || qa > pa || q < p)) ? 4u : 0u;
       }
     }
     dup = group8_or(dup);
@@ -567,7 +568,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       in_filt[f] = 1;
     }
   }
-  uint32_t F = 0, F0 = 0;                 // entries emitted so far; length of the first list
+  uint32_t F = 0;                         // entries emitted so far
   const uint32_t n_lists = c.stateful ? 2u : 1u;
   for (uint32_t list = 0; list < n_lists; ++list) {
     __syncthreads();
@@ -746,7 +747,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       keys_g[F + pos] = ((unsigned long long)acc << 32) | pred_p;
       ids_g[F + pos] = id;
       loc_g[F + pos] = (uint16_t)(v32 & 0xFFFFu);
-      if (list == 0 && pos < INDEX_MAX_F) { S.ids[pos] = id; S.pred[pos] = pred_p; S.acc[pos] = (uint16_t)acc; }   // first segment
+      if (F + pos < INDEX_MAX_F) { S.ids[F + pos] = id; S.pred[F + pos] = pred_p; S.acc[F + pos] = (uint16_t)acc; }   // first segment
     };
     if (!small) {
       uint32_t kept_so_far = 0;
@@ -785,19 +786,19 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       if (mine_kept && sidx == 0) emit(rank, a64, a32);
     }
     __syncthreads();
-    if (list == 0) F0 = Fl;
     F += Fl;
   }
   bool indexed = F > 0;
   bool counted = false;                       // has this CTA made its last allocation?
-  // index the lists segment by segment (INDEX_MAX_F positions each; almost always one)
+  // index the list -- the two lists of a state-aware catalog count as one, the Inactive entries
+  // behind the Active ones: "first position that meets both requirements, else the smallest
+  // distance at the lowest position" is all the index knows about order -- segment by segment
+  // (INDEX_MAX_F positions each; almost always one)
   if (indexed) {
-    const uint32_t segs0 = (F0 + INDEX_MAX_F - 1u) / INDEX_MAX_F;
-    const uint32_t nseg = segs0 + (F - F0 + INDEX_MAX_F - 1u) / INDEX_MAX_F, x0 = c.seg_base[t];
+    const uint32_t nseg = (F + INDEX_MAX_F - 1u) / INDEX_MAX_F, x0 = c.seg_base[t];
     for (uint32_t sg = 0; sg < nseg && indexed; ++sg) {
-      const uint32_t off = sg < segs0 ? sg * INDEX_MAX_F : F0 + (sg - segs0) * INDEX_MAX_F;
-      const uint32_t Fseg = min(INDEX_MAX_F, (sg < segs0 ? F0 : F) - off);
-      if (sg || F0 == 0) {                        // all but the first list's head: back from the task's region
+      const uint32_t off = sg * INDEX_MAX_F, Fseg = min(INDEX_MAX_F, F - off);
+      if (sg) {                                   // later segments: back from the task's region
         __syncthreads();
         for (uint32_t i = tid; i < Fseg; i += B) {
           const unsigned long long e = keys_g[off + i];
