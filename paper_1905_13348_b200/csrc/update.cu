@@ -413,31 +413,12 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   unsigned char *blk = c.image + base;
   unsigned char *slow = blk + BL.slow;
 
-  // From here on nothing depends on anything else: thread ranges take one table each.
+  // From here on nothing depends on anything else: thread ranges take one small table each.
   // [lo, lo + n) of the CTA's threads run `body(x)` for x = 0 .. count - 1.
   auto share = [&](uint32_t lo, uint32_t n, uint32_t count, auto body) {
     if (tid >= lo && tid < lo + n)
       for (uint32_t x = tid - lo; x < count; x += n) body(x);
   };
-
-  // T2: cell (r, k) = first position whose latency rank is < r and accuracy rank >= k
-  unsigned char *T2 = blk + BL.t2;
-  // four consecutive cells per step, stored as one word (the table is padded to a multiple of 4)
-  share(0, B / 2, ((Ks + 2u) * width + 3u) >> 2, [&](uint32_t q) {
-    uint32_t r = (q << 2) / width, k = (q << 2) - r * width, word = 0;
-#pragma unroll
-    for (uint32_t u = 0; u < 4; ++u) {
-      uint32_t pos = F;
-      if (r >= 1 && r <= Ks)
-        for (uint32_t w = 0; w < nw; ++w) {
-          const unsigned long long m = S.Lmask[r][w] & S.Amask[k][w];
-          if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
-        }
-      word |= pos << (8u * u);
-      if (++k == width) { k = 0; ++r; }
-    }
-    reinterpret_cast<uint32_t *>(T2)[q] = word;            // cells past the last row hold F
-  });
 
   // SLO records (see common.cuh)
   uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
@@ -509,6 +490,26 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   });
   uint32_t *Pd_g = reinterpret_cast<uint32_t *>(slow + SL.Pd);
   share(15 * B / 16, B / 16, Ks, [&](uint32_t i) { Pd_g[i] = S.Pd[i]; });
+
+  // T2: cell (r, k) = first position whose latency rank is < r and accuracy rank >= k.  The
+  // largest table: all threads, after their share of the small ones.
+  unsigned char *T2 = blk + BL.t2;
+  // four consecutive cells per step, stored as one word (the table is padded to a multiple of 4)
+  share(0, B, ((Ks + 2u) * width + 3u) >> 2, [&](uint32_t q) {
+    uint32_t r = (q << 2) / width, k = (q << 2) - r * width, word = 0;
+#pragma unroll
+    for (uint32_t u = 0; u < 4; ++u) {
+      uint32_t pos = F;
+      if (r >= 1 && r <= Ks)
+        for (uint32_t w = 0; w < nw; ++w) {
+          const unsigned long long m = S.Lmask[r][w] & S.Amask[k][w];
+          if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
+        }
+      word |= pos << (8u * u);
+      if (++k == width) { k = 0; ++r; }
+    }
+    reinterpret_cast<uint32_t *>(T2)[q] = word;            // cells past the last row hold F
+  });
 
   const uint32_t cb = ((BL.bitmap - BL.t2) >> 2) + CB_BIAS - acc_lo / ACC_WORD_BITS;
   const uint4 hdr = make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
