@@ -316,10 +316,12 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     uint32_t dup = 0;
     if (p < F) {
       const uint32_t pp = S.pred[p], pa = S.acc[p];
-      for (uint32_t q = sub; q < F; q += 8) {
+#pragma unroll 4
+      for (uint32_t q = sub; q < F; q += 8) {              // no branches: the trips' loads overlap
         const uint32_t qp = S.pred[q], qa = S.acc[q];
-        if (q < p) dup |= (qp == pp ? 1u : 0u) | (qa == pa ? 2u : 0u);
-        dup |= (qp <= pp && qa >= pa && (qp < pp || qa > pa || q < p)) ? 4u : 0u;
+        const uint32_t earlier = q < p;
+        dup |= (earlier & (uint32_t)(qp == pp)) | ((earlier & (uint32_t)(qa == pa)) << 1);
+        dup |= ((uint32_t)(qp <= pp) & (uint32_t)(qa >= pa) & ((uint32_t)(qp < pp) | (uint32_t)(qa > pa) | earlier)) << 2;
       }
     }
     dup = group8_or(dup);
@@ -334,8 +336,9 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     uint32_t cnt = 0;                                  // latency rank | accuracy rank << 16
     if (p < F) {
       const uint32_t pp = S.pred[p], pa = S.acc[p];
+#pragma unroll 4
       for (uint32_t q = sub; q < F; q += 8)
-        cnt += ((S.firstP[q] && S.pred[q] < pp) ? 1u : 0u) + ((S.firstA[q] && S.acc[q] < pa) ? 0x10000u : 0u);
+        cnt += ((uint32_t)S.firstP[q] & (uint32_t)(S.pred[q] < pp)) + (((uint32_t)S.firstA[q] & (uint32_t)(S.acc[q] < pa)) << 16);
     }
     cnt = group8_add(cnt);
     if (p < F && sub == 0) {
