@@ -5,6 +5,8 @@
 // Here a window's decisions are counted per variant (tally kernel), each variant's queue is
 // advanced by one window and its load-adjusted latency recomputed, and every task's list of
 // non-dominated variants is rebuilt in (cost, pred_lat, -acc, id) order (rebuild kernel).
+// On a state-aware catalog the same step moves the variants' life-cycle states with the load
+// (Section 4, state machine) and builds the Active and the Inactive list of every task.
 #include "common.cuh"
 
 namespace infaas {
@@ -744,7 +746,7 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
     __syncthreads();
     const uint32_t Fl = s_total;
 
-    // 4. compact into the task's region (scan order, behind the earlier list): keys and ids
+    // 4. into the task's region (scan order, behind the earlier list): keys, ids, local indices
     auto emit = [&](uint32_t pos, unsigned long long v64, uint32_t v32) {   // position pos of this list
       const uint32_t pred_p = (uint32_t)v64, acc = 10000u - (v32 >> 16);
       const uint32_t id = c.s_id[base + (v32 & 0xFFFFu)];
