@@ -724,20 +724,21 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
       // 3. prune.  In sorted order every dominator of p sits before p, and every earlier entry
       // q with pred_q <= pred_p and acc_q >= acc_p dominates p (its cost is not larger by the
       // sort, and it differs in some attribute or has the smaller id).
-      for (uint32_t p = tid; p < V; p += B) {
-        const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
+      // One entry per warp at a time: its 32 lanes scan the earlier entries 32 at a time and stop
+      // at the first chunk that holds a dominator (a survivor costs p / 32 trips of the whole
+      // warp instead of p trips of one lane).
+      for (uint32_t p = tid >> 5; p < V; p += B >> 5) {       // uniform per warp
         bool kp = p < Vl;
-        for (uint32_t q0 = 0; q0 < p && kp; q0 += 8) {     // groups of 8, exit between groups
-          bool dom = false;
-#pragma unroll
-          for (uint32_t j = 0; j < 8; ++j) {
-            const uint32_t q = min(q0 + j, p - 1);          // clamped repeats are harmless
-            dom |= (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
+        if (kp) {
+          const uint32_t pred_p = (uint32_t)k64[p], inv_p = k32[p] >> 16;
+          for (uint32_t q0 = 0; q0 < p; q0 += 32) {         // from p - 1 down: a dominator tends to cost
+            const uint32_t back = q0 + (tid & 31u);         // about as much as the entry itself
+            const uint32_t q = p - 1u - min(back, p - 1u);
+            const bool dom = back < p && (uint32_t)k64[q] <= pred_p && (k32[q] >> 16) <= inv_p;
+            if (__any_sync(0xFFFFFFFFu, dom)) { kp = false; break; }
           }
-          kp = !dom;
         }
-        keep[p] = kp;
-        my_kept += kp;
+        if ((tid & 31u) == 0) { keep[p] = kp; my_kept += kp; }
       }
     }
     __syncthreads();
