@@ -190,7 +190,7 @@ struct IndexScratch {          // shared memory used while building one task's i
   unsigned char idxP[256], idxA[256], firstP[256], firstA[256], on_stair[256];
   uint32_t bcnt[256], bthr[256];    // per SLO bucket: distinct latencies inside it, one of them
   uint32_t wbits[256];              // per bitmap word: the accuracies present
-  unsigned long long Lmask[256][4], Amask[256][4];   // positions by latency rank < r / accuracy rank >= k
+  unsigned long long Lmask[4][256], Amask[4][256];   // [word][rank]: positions by latency rank < r / accuracy rank >= k
   // per latency rank: the most accurate entry (acc << 16 | 0xFFFF - position, 0 = none) and
   // 1 + position of its stair entry (0 = none); per accuracy rank: the fastest entry
   // (pred << 32 | position, ~0 = none); then their running maximum / minimum / count
@@ -404,7 +404,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
       const bool in = which ? S.idxA[p] >= rk : S.idxP[p] < rk;
       m |= (unsigned long long)in << (p & 63u);
     }
-    (which ? S.Amask : S.Lmask)[rk][w] = m;
+    (which ? S.Amask : S.Lmask)[w][rk] = m;
   }
 
   if (tid == 0) {
@@ -499,21 +499,17 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   // T2: cell (r, k) = first position whose latency rank is < r and accuracy rank >= k.  The
   // largest table: all threads, after their share of the small ones.
   unsigned char *T2 = blk + BL.t2;
-  // four consecutive cells per step, stored as one word (the table is padded to a multiple of 4)
-  share(0, B, ((Ks + 2u) * width + 3u) >> 2, [&](uint32_t q) {
-    uint32_t r = (q << 2) / width, k = (q << 2) - r * width, word = 0;
-#pragma unroll
-    for (uint32_t u = 0; u < 4; ++u) {
-      uint32_t pos = F;
-      if (r >= 1 && r <= Ks)
-        for (uint32_t w = 0; w < nw; ++w) {
-          const unsigned long long m = S.Lmask[r][w] & S.Amask[k][w];
-          if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
-        }
-      word |= pos << (8u * u);
-      if (++k == width) { k = 0; ++r; }
-    }
-    reinterpret_cast<uint32_t *>(T2)[q] = word;            // cells past the last row hold F
+  // consecutive lanes take consecutive cells: the same r (a broadcast) and consecutive k, which
+  // the word-major masks serve without bank conflicts
+  share(0, B, (Ks + 2u) * width, [&](uint32_t cell) {
+    const uint32_t r = cell / width, k = cell - r * width;
+    uint32_t pos = F;
+    if (r >= 1 && r <= Ks)
+      for (uint32_t w = 0; w < nw; ++w) {
+        const unsigned long long m = S.Lmask[w][r] & S.Amask[w][k];
+        if (m) { pos = 64u * w + (uint32_t)__ffsll((long long)m) - 1u; break; }
+      }
+    T2[cell] = (unsigned char)pos;
   });
 
   const uint32_t cb = ((BL.bitmap - BL.t2) >> 2) + CB_BIAS - acc_lo / ACC_WORD_BITS;
