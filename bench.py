@@ -34,12 +34,12 @@ FALLBACK_HBM_GBS = 6650.0
 # workload, from the ncu capture summarised in profiles/select_kernel_C3.md, per query (part of
 # the decisions is still in L2 when the kernel ends, hence below 12 B).  Set to None when the
 # kernel changes until the counters are taken again.
-NCU_TRAFFIC_BYTES_PER_QUERY = (134.55e6 + 26.53e6) / (1 << 24)
+NCU_TRAFFIC_BYTES_PER_QUERY = (134.55e6 + 28.25e6) / (1 << 24)
 # From the same capture: warp-instructions executed and shared-memory wavefronts (one per
 # clock and SM at most) per query, for the two on-chip limits the kernel sits closer to than
 # to HBM.  Same rule as above when the kernel changes.
 NCU_WARP_INSTR_PER_QUERY = 41.39e6 / (1 << 24)
-NCU_SMEM_WAVEFRONTS_PER_QUERY = 10.34e6 / (1 << 24)
+NCU_SMEM_WAVEFRONTS_PER_QUERY = 10.38e6 / (1 << 24)
 SM_COUNT, ISSUE_PER_SM_CLK = 148, 4
 
 
