@@ -41,6 +41,8 @@ NCU_TRAFFIC_BYTES_PER_QUERY = (134.55e6 + 28.25e6) / (1 << 24)
 NCU_WARP_INSTR_PER_QUERY = 41.39e6 / (1 << 24)
 NCU_SMEM_WAVEFRONTS_PER_QUERY = 10.38e6 / (1 << 24)
 SM_COUNT, ISSUE_PER_SM_CLK = 148, 4
+# end-to-end leg: shares of the batch per chunk (the rest is the last chunk)
+E2E_CHUNK_SHARES = (0.36, 0.26, 0.18, 0.11, 0.06)
 
 
 def parse_args():
@@ -356,21 +358,23 @@ def run_ours(args):
 def e2e_leg(P, cat, w, dev, update, steps, world, dist):
     """Same step with HOST inputs and outputs: pinned host arrays are copied to the device,
     decided, and the decisions copied back, all inside the timed region.  The work is chunked
-    and pipelined over three streams so that upload, kernels and download overlap."""
+    and pipelined over three streams so that upload, kernels and download overlap; every step's
+    selection still sees the load update of the step before."""
     import torch
     n = w.n_queries
     h_task = torch.from_numpy(w.task.view(np.int16)).pin_memory()
     h_slo = torch.from_numpy(w.slo_us.view(np.int32)).pin_memory()
     h_acc = torch.from_numpy(w.min_acc_bp.view(np.int16)).pin_memory()
     h_dec = torch.empty(n, dtype=torch.int32).pin_memory()
-    d_task = torch.empty(n, dtype=torch.int16, device=dev)
-    d_slo = torch.empty(n, dtype=torch.int32, device=dev)
-    d_acc = torch.empty(n, dtype=torch.int16, device=dev)
-    d_dec = torch.empty(n, dtype=torch.int32, device=dev)
+    # two sets of device arrays: the upload of one step runs while the previous step's last
+    # chunk is still being decided, downloaded and tallied
+    dsets = [(torch.empty(n, dtype=torch.int16, device=dev), torch.empty(n, dtype=torch.int32, device=dev),
+              torch.empty(n, dtype=torch.int16, device=dev), torch.empty(n, dtype=torch.int32, device=dev))
+             for _ in range(2)]
     # few, large copies (each costs some 4-10 us of set-up on top of its bytes), shrinking
     # towards the end so that little is left to do after the last upload
     bounds, lo = [], 0
-    for share in (0.36, 0.26, 0.18, 0.11, 0.06):
+    for share in E2E_CHUNK_SHARES:
         hi = min(n, lo + max(8, int(n * share) // 8 * 8))
         if hi > lo:
             bounds.append((lo, hi))
@@ -378,37 +382,43 @@ def e2e_leg(P, cat, w, dev, update, steps, world, dist):
     if lo < n:
         bounds.append((lo, n))
     up, comp, down = (torch.cuda.Stream(dev) for _ in range(3))
-    ev_up = [torch.cuda.Event() for _ in bounds]
-    ev_sel = [torch.cuda.Event() for _ in bounds]
+    ev_up = [[torch.cuda.Event() for _ in bounds] for _ in range(2)]
+    ev_sel = [[torch.cuda.Event() for _ in bounds] for _ in range(2)]
+    ev_updated = [torch.cuda.Event() for _ in range(2)]      # the step that used this set has been tallied
+    ev_down = [torch.cuda.Event() for _ in range(2)]         # ... and its decisions are on the host
     main = torch.cuda.current_stream()
+    for st in (up, comp, down):
+        st.wait_stream(main)
+    for s_ in range(2):
+        ev_updated[s_].record(comp)
+        ev_down[s_].record(down)
+    host = [tuple(x[lo:hi] for x in (h_task, h_slo, h_acc, h_dec)) for lo, hi in bounds]
+    devv = [[tuple(x[lo:hi] for x in dset) for lo, hi in bounds] for dset in dsets]
+    count = [0]
 
-    views = [tuple(x[lo:hi] for x in (h_task, h_slo, h_acc, d_task, d_slo, d_acc, d_dec, h_dec)) for lo, hi in bounds]
-
-    def body(main):
-        # upload, selection and download each on a stream of their own, chained per chunk by
-        # events: the upload (the longest of the three) never waits for anything
-        up.wait_stream(main)
-        comp.wait_stream(main)
-        down.wait_stream(main)
-        for i, (ht, hs, ha, dt_, ds, da, dd, hd) in enumerate(views):
+    def step():
+        # upload, selection (+ the load update, which the next step's selection must see) and
+        # download each on a stream of their own, chained per chunk by events
+        k = count[0] & 1
+        count[0] += 1
+        up.wait_event(ev_updated[k])           # the inputs of the step before last have been read
+        comp.wait_event(ev_down[k])            # ... and its decisions copied out
+        for i, (ht, hs, ha, hd) in enumerate(host):
+            dt_, ds, da, dd = devv[k][i]
             with torch.cuda.stream(up):
                 dt_.copy_(ht, non_blocking=True)
                 ds.copy_(hs, non_blocking=True)
                 da.copy_(ha, non_blocking=True)
-                ev_up[i].record(up)
-            comp.wait_event(ev_up[i])
+                ev_up[k][i].record(up)
+            comp.wait_event(ev_up[k][i])
             P.infaas_select_batch(cat, dt_, ds, da, dd, stream=comp)
-            ev_sel[i].record(comp)
-            down.wait_event(ev_sel[i])
+            ev_sel[k][i].record(comp)
+            down.wait_event(ev_sel[k][i])
             with torch.cuda.stream(down):
                 hd.copy_(dd, non_blocking=True)
-        main.wait_stream(up)
-        main.wait_stream(comp)
-        main.wait_stream(down)
-        update(d_dec, main)
-
-    def step():
-        body(main)
+        ev_down[k].record(down)
+        update(dsets[k][3], comp)
+        ev_updated[k].record(comp)
 
     for _ in range(3):
         step()
@@ -427,8 +437,9 @@ def e2e_leg(P, cat, w, dev, update, steps, world, dist):
     return {"value": world * n * steps / dt, "unit": UNIT, "h2d_bytes_per_step": 8 * n,
             "d2h_bytes_per_step": 4 * n, "ms_per_step": 1e3 * dt / steps, "steps": steps,
             "how": f"pinned host -> device copies, select and download per chunk ({len(bounds)} chunks of "
-                   "decreasing size; upload / select / download streams chained by events), one load "
-                   "update; host wall clock around synchronize"}
+                   "decreasing size; upload / select + load update / download streams chained by events; "
+                   "two sets of device arrays, so a step's upload overlaps the end of the step before); "
+                   "host wall clock around synchronize"}
 
 
 def windowed_leg(P, cat, w, inp, d_dec, world):
