@@ -529,15 +529,8 @@ static_assert(REBUILD_THREADS == 1024 && SLO_BUCKETS == 256, "thread ranges of b
 constexpr uint32_t RANK_SORT_MAX = 512;   // tasks up to this size are sorted by counting smaller keys
 
 __global__ void __launch_bounds__(REBUILD_THREADS)
-rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us) {
+rebuild_kernel(DeviceCatalog c, int advance, uint32_t window_us) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // small tasks have, in front of the sort buffers, the attributes packed for the prune (kept a
-  // plain offset from the shared array so that the loads stay shared-memory loads)
-  const bool small = sort_n <= RANK_SORT_MAX;
-  uint4 *attr = reinterpret_cast<uint4 *>(smem_raw);
-  unsigned long long *k64 = reinterpret_cast<unsigned long long *>(smem_raw + (small ? 16u * sort_n : 0u));   // cost<<32 | pred
-  uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + sort_n);                    // inv_acc<<16 | local
-  unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + sort_n);         // 1 = non-dominated
   __shared__ uint32_t warp_sums[32];
   __shared__ uint32_t s_total, s_inlist, s_ncand, s_nnew;
   __shared__ uint16_t filt[RANK_SORT_MAX], cand[RANK_SORT_MAX], newc[RANK_SORT_MAX];   // small tasks: filter set,
@@ -551,6 +544,14 @@ rebuild_kernel(DeviceCatalog c, uint32_t sort_n, int advance, uint32_t window_us
   // sort size for this task: the power of two that holds it (tasks differ in size)
   uint32_t P = 1;
   while (P < V) P <<= 1;
+  // small tasks (each task decides for itself) have, in front of the sort buffers, the attributes
+  // packed for the prune (kept a plain offset from the shared array so that the loads stay
+  // shared-memory loads)
+  const bool small = P <= RANK_SORT_MAX;
+  uint4 *attr = reinterpret_cast<uint4 *>(smem_raw);
+  unsigned long long *k64 = reinterpret_cast<unsigned long long *>(smem_raw + (small ? 16u * P : 0u));   // cost<<32 | pred
+  uint32_t *k32 = reinterpret_cast<uint32_t *>(k64 + P);                         // inv_acc<<16 | local
+  unsigned char *keep = reinterpret_cast<unsigned char *>(k32 + P);              // 1 = non-dominated
 
   // A state-aware catalog has two lists per task: Active variants keyed (cost, pred, 10000-acc,
   // id), then Inactive ones keyed by their combined loading + inference latency, which takes
@@ -872,9 +873,12 @@ cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t
                            cudaStream_t stream) {
   uint32_t P = 1;
   while (P < c.max_task_variants) P <<= 1;
-  // small tasks: room for the packed attributes (16 bytes per entry)
-  size_t smem = (size_t)P * 13 + (P <= RANK_SORT_MAX ? (size_t)P * 16 + 32 : 0);
-  rebuild_kernel<<<c.n_tasks, REBUILD_THREADS, smem, stream>>>(c, P, advance_queues ? 1 : 0, window_us);
+  // sort buffers of the largest task (13 bytes per padded entry); a small task needs 29 bytes per
+  // padded entry (packed attributes in front), at most for RANK_SORT_MAX entries
+  const uint32_t Ps = P < RANK_SORT_MAX ? P : RANK_SORT_MAX;
+  size_t smem = (size_t)P * 13;
+  if (smem < (size_t)Ps * 29 + 32) smem = (size_t)Ps * 29 + 32;
+  rebuild_kernel<<<c.n_tasks, REBUILD_THREADS, smem, stream>>>(c, advance_queues ? 1 : 0, window_us);
   return cudaGetLastError();
 }
 
