@@ -73,3 +73,17 @@ def test_binding_fails_loudly_without_device():
     import paper_1905_13348_b200 as P
     with pytest.raises(P.InfaasError):
         P.infaas_catalog_load(W.make("C1").rows, 1)
+
+
+def test_binding_constants_match_the_header():
+    text = open(os.path.join(ROOT, "include", "infaas.h")).read()
+    defs = {m.group(1): int(m.group(2).rstrip("u"), 0)
+            for m in re.finditer(r"#define\s+(INFAAS_[A-Z_]+)\s+\(?(-?(?:0x[0-9A-Fa-f]+|\d+)u?)\)?", text)}
+    from paper_1905_13348_b200 import binding as b
+    assert defs["INFAAS_NO_FEASIBLE"] == b.NO_FEASIBLE and defs["INFAAS_INVALID"] == b.INVALID
+    assert [defs[f"INFAAS_STATE_{n}"] for n in ("INACTIVE", "ACTIVE", "OVERLOADED", "INTERFERED")] == \
+        [b.STATE_INACTIVE, b.STATE_ACTIVE, b.STATE_OVERLOADED, b.STATE_INTERFERED]
+    assert defs["INFAAS_AUTOSCALE_NONE"] == b.AUTOSCALE_NONE and defs["INFAAS_AUTOSCALE_ESCALATE"] == b.AUTOSCALE_ESCALATE
+    assert sorted(b.EXPORTS) == sorted(n for n in declared_functions())
+    codes = sorted(v for k, v in defs.items() if k.startswith("INFAAS_E_"))
+    assert codes == list(range(-11, 0))
