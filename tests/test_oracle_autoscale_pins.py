@@ -183,3 +183,29 @@ def test_need_is_rounded_up():
     for inst, want in ((336_666_666, (0, 1)), (336_666_667, (AUTOSCALE_NONE, 0)), (336_666_000, (0, 667))):
         v, d = autoscale_step(rows, 1, [1], [inst], [0], [2**32 - 1], 3, 101, 0)
         assert (int(v[0]), int(d[0])) == want
+
+
+# -- monotone in the load and in what already runs -------------------------------------------------
+def test_more_load_never_needs_less_and_more_instances_never_need_more():
+    rng = np.random.default_rng(43)
+    nv = 40
+    rows = _rows([0] * nv, rng.choice([1, 2, 4, 8], nv), rng.integers(2000, 200000, nv), rng.integers(1, 50, nv), [3] * nv)
+    inst = np.zeros(nv, np.uint32); inst[5] = 2
+    load = np.zeros(nv, np.uint32)
+    prev = 0
+    for served in (0, 10, 100, 1000, 10000, 100000):
+        count = np.zeros(nv, np.uint32); count[5] = served
+        v, d = autoscale_step(rows, 1, count, inst, load, [10**6], 10**6, 105, 0)
+        cost = 0 if int(v[0]) >= AUTOSCALE_ESCALATE else int(rows["cost"][int(v[0])]) * int(d[0])
+        assert cost >= prev
+        prev = cost
+    assert prev > 0
+    count = np.zeros(nv, np.uint32); count[5] = 100000
+    prev = None
+    for n in (1, 2, 8, 64, 10**6):
+        inst[5] = n
+        v, d = autoscale_step(rows, 1, count, inst, load, [10**6], 10**6, 105, 0)
+        cost = 0 if int(v[0]) >= AUTOSCALE_ESCALATE else int(rows["cost"][int(v[0])]) * int(d[0])
+        assert prev is None or cost <= prev
+        prev = cost
+    assert prev == 0 and int(v[0]) == AUTOSCALE_NONE

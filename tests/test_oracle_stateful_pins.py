@@ -190,3 +190,40 @@ def test_inactive_ties_and_saturation():
     assert int(s.select([0], [2**32 - 1], [7200])[0]) == 2
     assert int(s.select([0], [2**32 - 2], [7200])[0]) == (NO_FEASIBLE_BIT | 2)
     assert int(s.select([0], [2**32 - 2], [0])[0]) == 3
+
+
+# -- permuting the catalog rows (ids, states and loading latencies carried along) -----------------
+def test_row_permutation_equivariance_stateful():
+    w = W.make("C2", n_queries=4000)
+    rng = np.random.default_rng(6)
+    state = _random_states(rng, w.n_variants, (0.5, 0.3, 0.1, 0.1))
+    load = rng.integers(0, 200_000, w.n_variants).astype(np.uint32)
+    d0 = StatefulOracleCatalog(w.rows, w.n_tasks, state, load).select(w.task, w.slo_us, w.min_acc_bp, 3)
+    perm = rng.permutation(w.n_variants)
+    d1 = StatefulOracleCatalog(w.rows[perm], w.n_tasks, state[perm], load[perm]).select(w.task, w.slo_us, w.min_acc_bp)
+    assert np.array_equal(d1 == INVALID, d0 == INVALID)
+    ok = d0 != INVALID
+    assert np.array_equal(d1[ok] & NO_FEASIBLE_BIT, d0[ok] & NO_FEASIBLE_BIT)
+    r0, r1 = w.rows[d0[ok] & 0x7FFFFFFF], w.rows[perm][d1[ok] & 0x7FFFFFFF]
+    for k in ("cost", "lat_us", "acc_bp", "batch", "queued"):   # the same variant up to id ties
+        assert np.array_equal(r0[k], r1[k])
+    assert np.array_equal(state[d0[ok] & 0x7FFFFFFF], state[perm][d1[ok] & 0x7FFFFFFF])
+
+
+# -- loading a variant (Inactive -> Active) never turns a served query into an unserved one ------
+def test_activation_is_monotone():
+    w = W.make("C2", n_queries=4000)
+    rng = np.random.default_rng(7)
+    state = _random_states(rng, w.n_variants, (0.7, 0.2, 0.05, 0.05))
+    load = rng.integers(1000, 300_000, w.n_variants).astype(np.uint32)
+    d0 = StatefulOracleCatalog(w.rows, w.n_tasks, state, load).select(w.task, w.slo_us, w.min_acc_bp, 3)
+    state2 = state.copy()
+    flip = (state == INACTIVE) & (rng.random(w.n_variants) < 0.5)
+    state2[flip] = ACTIVE
+    d1 = StatefulOracleCatalog(w.rows, w.n_tasks, state2, load).select(w.task, w.slo_us, w.min_acc_bp, 3)
+    served0, served1 = (d0 >> 31) == 0, (d1 >> 31) == 0
+    assert np.all(served1[served0]) and served1.sum() > served0.sum()
+    # and a query that an Active variant already served is still served by an Active one, no dearer
+    was_active = served0 & (state[d0 & 0x7FFFFFFF] == ACTIVE)
+    assert np.all(state2[d1[was_active]] == ACTIVE)
+    assert np.all(w.rows["cost"][d1[was_active]].astype(np.int64) <= w.rows["cost"][d0[was_active]].astype(np.int64))
