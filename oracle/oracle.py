@@ -15,8 +15,10 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "infaas_oracle.cpp")
-_LIB = os.path.join(_HERE, "libinfaas_oracle.so")
+# INFAAS_ORACLE_SRC: another copy of the source to build and load instead (the test that plants
+# mistakes in a scratch copy and checks that the pins notice uses it).
+_SRC = os.environ.get("INFAAS_ORACLE_SRC") or os.path.join(_HERE, "infaas_oracle.cpp")
+_LIB = os.path.join(os.path.dirname(os.path.abspath(_SRC)), "libinfaas_oracle.so")
 _lib = None
 
 NO_FEASIBLE_BIT = 0x80000000

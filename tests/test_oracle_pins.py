@@ -157,6 +157,42 @@ def test_tie_break_order():
     assert int(_select(rows, 1, [0], [1000], [0])[0]) == 0     # predicted, not profiled, latency
 
 
+# -- ties between nearest misses at equal distance: cost, then predicted latency, then accuracy,
+#    then id (the order of the feasible branch, after the distance).  Every case pits two
+#    criteria against each other, so that a key with two fields swapped answers differently. --
+def test_nearest_miss_tie_break_order():
+    def miss(rows, slo, acc):
+        d = int(_select(rows, 1, [0], [slo], [acc])[0])
+        assert d & NO_FEASIBLE_BIT
+        return d & 0x7FFFFFFF
+    # both meet the SLO and miss the accuracy by one basis point (d = 100 each):
+    # id0 is slower and cheaper, id1 faster and dearer -> cost decides
+    rows = rows_from([0, 0], [1, 1], [20, 10], [7000, 7000], [1, 2])
+    assert miss(rows, 100, 7001) == 0
+    rows = rows_from([0, 0], [1, 1], [10, 20], [7000, 7000], [2, 1])
+    assert miss(rows, 100, 7001) == 1
+    # one misses the SLO by 1 us (d = 10^4), the other the accuracy by 100 bp at slo 100
+    # (d = 10^4): id0 slower and cheaper -> cost decides, not latency
+    rows = rows_from([0, 0], [1, 1], [101, 50], [7000, 6900], [1, 2])
+    assert miss(rows, 100, 7000) == 0
+    rows = rows_from([0, 0], [1, 1], [50, 101], [6900, 7000], [2, 1])
+    assert miss(rows, 100, 7000) == 1
+    # a strictly smaller distance beats a lower cost
+    rows = rows_from([0, 0], [1, 1], [101, 50], [7000, 6901], [1, 9])      # d = 10000, 9900
+    assert miss(rows, 100, 7000) == 1
+    rows = rows_from([0, 0], [1, 1], [101, 50], [7000, 6899], [9, 1])      # d = 10000, 10100
+    assert miss(rows, 100, 7000) == 0
+    # equal distance and cost: the faster one, although it is the less accurate and has the higher id
+    rows = rows_from([0, 0], [1, 1], [101, 60], [7000, 6900], [3, 3])
+    assert miss(rows, 100, 7000) == 1
+    # equal distance, cost and latency (both miss the SLO only): higher accuracy, then lower id
+    rows = rows_from([0, 0, 0], [1, 1, 1], [150, 150, 150], [7100, 7300, 7300], [3, 3, 3])
+    assert miss(rows, 100, 7000) == 1
+    # predicted latency, not the profiled one, enters both the distance and the tie
+    rows = rows_from([0, 0], [1, 1], [30, 50], [7000, 7000], [4, 4], [1, 0])   # pred 60, 50
+    assert miss(rows, 100, 7001) == 1
+
+
 # -- P5: permuting the catalog rows (ids carried along) permutes the answers ---------------
 def test_row_permutation_equivariance():
     w = W.make("C2", n_queries=5000)

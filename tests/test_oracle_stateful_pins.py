@@ -148,6 +148,38 @@ def test_suggestion_prefers_active_on_equal_distance():
     assert int(s.select([0], [100], [7000])[0]) == INVALID
 
 
+# -- equal distance inside one class: Active by (cost, latency, accuracy, id), Inactive by
+#    (combined latency, accuracy, id); every case sets two criteria against each other ---------
+def test_suggestion_tie_break_order_inside_a_class():
+    def miss(rows, state, load, slo, acc):
+        d = int(StatefulOracleCatalog(rows, 1, state, load).select([0], [slo], [acc])[0])
+        assert d & NO_FEASIBLE_BIT
+        return d & 0x7FFFFFFF
+    A, I = ACTIVE, INACTIVE
+    # Active pair, both miss the accuracy by 1 bp: slower and cheaper wins (cost before latency)
+    rows = rows_from([0, 0], [1, 1], [20, 10], [7000, 7000], [1, 2])
+    assert miss(rows, [A, A], [0, 0], 100, 7001) == 0
+    # Active pair, one over the SLO by 1 us, one under the accuracy by 100 bp at slo 100
+    rows = rows_from([0, 0], [1, 1], [101, 50], [7000, 6900], [1, 2])
+    assert miss(rows, [A, A], [0, 0], 100, 7000) == 0
+    rows = rows_from([0, 0], [1, 1], [50, 101], [6900, 7000], [2, 1])
+    assert miss(rows, [A, A], [0, 0], 100, 7000) == 1
+    # the same pair Inactive: the quicker one wins although it is dearer and less accurate
+    rows = rows_from([0, 0], [1, 1], [101, 50], [7000, 6900], [1, 2])
+    assert miss(rows, [I, I], [0, 0], 100, 7000) == 1
+    # ... through the loading latency too: 40 + 61 against 30 + 20
+    rows = rows_from([0, 0], [1, 1], [40, 30], [7000, 6900], [1, 2])
+    assert miss(rows, [I, I], [61, 20], 100, 7000) == 1
+    # Inactive, equal distance and combined latency: higher accuracy before lower id, cost ignored
+    rows = rows_from([0, 0, 0], [1, 1, 1], [150, 100, 150], [7100, 7300, 7300], [1, 9, 9])
+    assert miss(rows, [I, I, I], [0, 50, 0], 100, 7000) == 1
+    # Inactive pair, both miss the accuracy by 1 bp at the same distance: lower combined latency
+    # first, although the other one is the more accurate... which would change the distance, so
+    # equal accuracy here and the combined latency alone decides (cost the other way round)
+    rows = rows_from([0, 0], [1, 1], [20, 10], [7000, 7000], [1, 2])
+    assert miss(rows, [I, I], [0, 0], 100, 7001) == 1
+
+
 # -- state transitions at the end of a window: closed form under constant arrivals --------------
 def test_state_transitions_closed_form():
     #         id0        id1       id2         id3

@@ -38,6 +38,34 @@ def test_against_sorting(seed):
     assert [int(x) for x in got] == [plain(rows, iv, iw, il, hw, ut, int(d)) for d in dec]
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_against_sorting_mostly_unloaded(seed):
+    """Most variants have no instance, so the choice falls to the utilisation rule, with few
+    distinct utilisations: equal ones must go to the lower worker id."""
+    rng = np.random.default_rng(500 + seed)
+    nv, nw = int(rng.integers(6, 20)), int(rng.integers(3, 12))
+    rows = _rows(nv, rng.integers(0, 2, nv))
+    loaded = rng.choice(nv, 2, replace=False)
+    iv, iw, il = np.repeat(loaded, 2), rng.integers(0, nw, 4), rng.integers(0, 3, 4)
+    hw, ut = rng.integers(0, 2, nw), rng.integers(0, 2, nw)
+    dec = np.arange(nv, dtype=np.uint32)
+    got = assign_workers(rows, iv, iw, il, hw, ut, dec)
+    assert [int(x) for x in got] == [plain(rows, iv, iw, il, hw, ut, int(d)) for d in dec]
+
+
+def test_equal_utilisation_goes_to_the_lowest_worker_id():
+    rows = _rows(2, [0, 1])
+    none = np.zeros(0, np.uint32)
+    # three workers with the variant's hardware and the same utilisation -> worker 0
+    assert int(assign_workers(rows, none, none, none, [0, 0, 0], [5, 5, 5], [0])[0]) == 0
+    # the first two lack the hardware; of the equal rest the lowest id
+    assert int(assign_workers(rows, none, none, none, [0, 0, 1, 1, 1], [1, 1, 7, 7, 7], [1])[0]) == 2
+    # a lower utilisation later in the table still wins
+    assert int(assign_workers(rows, none, none, none, [0, 0, 0], [5, 5, 4], [0])[0]) == 2
+    # equal loads of a variant's instances -> lower worker id, whatever the table order
+    assert int(assign_workers(rows, [0, 0, 0], [2, 1, 3], [4, 4, 4], [0] * 4, [0] * 4, [0])[0]) == 1
+
+
 def test_special_cases_reduce_to_argmin():
     rng = np.random.default_rng(42)
     nv, nw = 50, 40
