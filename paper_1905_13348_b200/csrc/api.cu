@@ -66,6 +66,14 @@ inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// IEEE-754 single-precision pattern of x (> 0) converted toward zero, as the kernels compute it.
+inline uint32_t float_bits_rz(uint32_t x) {
+  uint32_t e = 31;
+  while (!(x >> e)) --e;
+  const uint32_t mant = (uint32_t)(((uint64_t)x << (31 - e)) >> 8) & 0x7FFFFFu;
+  return ((e + 127u) << 23) | mant;
+}
+
 // Re-reads the image size from the device and decides how much shared memory the selection
 // kernel asks for: all of it while the image fits (it may grow or shrink between two such
 // refreshes without a change of plan), none for the image if it does not -- the kernel
@@ -112,6 +120,7 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
 
   // ---- validate and bucket by task (stable: ascending id inside a task) ----
   std::vector<uint32_t> task_off(n_tasks + 1, 0);
+  uint32_t acc_min = 10000, acc_max = 0, lat_min = 0xFFFFFFFFu;
   for (uint32_t v = 0; v < n_variants; ++v) {
     const infaas_variant &r = rows[v];
     if (r.task >= n_tasks) return INFAAS_E_BAD_TASK;
@@ -119,7 +128,13 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
     if (r.lat_us == 0) return INFAAS_E_BAD_LAT;
     if (r.acc_bp > 10000 || r.reserved != 0) return INFAAS_E_BAD_ACC;
     task_off[r.task + 1]++;
+    if (r.acc_bp < acc_min) acc_min = r.acc_bp;
+    if (r.acc_bp > acc_max) acc_max = r.acc_bp;
+    if (r.lat_us < lat_min) lat_min = r.lat_us;
   }
+  // the window of accuracies every bitmap of the index covers: whole words of 24 basis points
+  const uint32_t acc_lo = acc_min / infaas::ACC_WORD_BITS * infaas::ACC_WORD_BITS;
+  const uint32_t nbw = (acc_max + 1u - acc_lo) / infaas::ACC_WORD_BITS + 1u;
   uint32_t max_task = 0;
   for (uint32_t t = 0; t < n_tasks; ++t) {
     if (task_off[t + 1] > max_task) max_task = task_off[t + 1];
@@ -158,14 +173,14 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   // ---- one arena, carved into 256-byte aligned arrays ----
   // lists longer than the index supports are cut into segments; every segment but a task's
   // first needs a header and parameters outside the image
-  uint64_t worst_image = infaas::image_var_offset(n_tasks);
+  uint64_t worst_image = infaas::image_var_offset(n_tasks, nbw);
   std::vector<uint32_t> seg_base(n_tasks + 1, 0);
   for (uint32_t t = 0; t < n_tasks; ++t) {
     const uint32_t V = task_off[t + 1] - task_off[t];
     // a state-aware catalog has two lists per task (V entries together): one segment more
     const uint32_t segs = (V + infaas::INDEX_MAX_F - 1) / infaas::INDEX_MAX_F + 1;
     seg_base[t + 1] = seg_base[t] + segs - 1;
-    worst_image += (uint64_t)segs * infaas::block_capacity(V);
+    worst_image += (uint64_t)segs * infaas::block_capacity(V, nbw);
   }
   const uint32_t n_extra = seg_base[n_tasks];
   if (worst_image > 0xFFFFFFF0ull) { delete c; return INFAAS_E_TOO_LARGE; }
@@ -252,6 +267,9 @@ int infaas_catalog_load(const infaas_variant *rows, uint32_t n_variants, uint32_
   d.image = base + o_image;
   d.image_capacity = (uint32_t)worst_image;
   d.image_hdr = reinterpret_cast<uint32_t *>(base + o_hdr);
+  d.acc_lo = acc_lo;
+  d.nbw = nbw;
+  d.lat_code_lo = float_bits_rz(lat_min) >> 16;
   d.counters = reinterpret_cast<unsigned long long *>(base + o_counters);
   d.alloc_ctr = reinterpret_cast<unsigned long long *>(base + o_rebuild);
   d.err = reinterpret_cast<uint32_t *>(base + o_err);

@@ -32,41 +32,37 @@ namespace infaas {
 //
 // r comes from one record of a table of SLO_BUCKETS records per task.  The bucket of an
 // SLO is  j = clamp((bits(slo) >> S) - bmin, 0, 255)  with bits(x) = the IEEE-754 pattern
-// of x converted to float toward zero (a monotone, roughly logarithmic code) and S = 16..23
-// chosen per task.  A record is  R << 24 | C  and  r = (record + (slo & 0xFFFFFF)) >> 24:
+// of x converted to float toward zero (a monotone, roughly logarithmic code) and one S = 16..23
+// and bmin for the whole catalog.  A record is  R << 24 | C  and
+// r = (record + (slo & 0xFFFFFF)) >> 24:
 //   - no distinct latency inside the bucket: R = the rank there, C = 0 (never carries);
 //   - one latency `thr` inside it, and all SLOs of the bucket agree in their top byte:
 //     R = rank below, C = 0xFFFFFF - ((thr - 1) & 0xFFFFFF), so the add carries into R
 //     exactly when slo >= thr;
 //   - otherwise R = Ks + 1, C = 0: row Ks + 1 of T2 holds only F, which sends the query to
 //     the exact slow path.
-// The buckets cover the list's latencies up to the largest SLO any batch has asked for so
-// far (kept as a bit mask, at least SLO_CAP_FLOOR_US); larger latencies share bucket 255.
+// The buckets run from the smallest profiled latency of the catalog (a predicted latency is
+// never below it) up to the largest SLO any batch has asked for so far (kept as a bit mask,
+// at least SLO_CAP_FLOOR_US); larger latencies share bucket 255.  The rebuild kernel derives
+// S and bmin from these two and publishes them beside the image size.
 // k comes from a bitmap over accuracy values with running popcounts (24 bitmap bits and an
-// 8-bit prefix count per word), exact at one basis point.
+// 8-bit prefix count per word), exact at one basis point.  Every bitmap covers the same
+// window of accuracies, that of the whole catalog (fixed at load: acc_lo, a multiple of 24,
+// and nbw words), so the word an accuracy falls into does not depend on the task.
 //
 // Image (what the selection kernel stages in shared memory):
-//   hdr    (n_tasks + 1) x 128 bytes: 8 identical copies of a 16-byte header per task, so
-//          that the 8 lanes served by one shared-memory wavefront never collide; entry
-//          n_tasks serves queries whose task is out of range
+//   hdr    (n_tasks + 1) u32, one per task: t2_off / 4 | (Ka + 1) << 24; entry n_tasks serves
+//          queries whose task is out of range; padded to 128 bytes
 //   rec    (n_tasks + 1) x SLO_BUCKETS u32 records
+//   bitmap (n_tasks + 1) x nbw u32: the accuracy bitmaps of the tasks' first segments
 //   dummy  64 bytes (what tasks without an index point at: every query of theirs reads
 //          "none" and goes to the slow path)
-//   var    per-task blocks, each 64-byte aligned:
-//          ids   u32[F + 1] in REVERSE order: ids[p] sits at t2_off - 4 - 4p (t2_off is a
-//                multiple of 16), and the slot
+//   var    per-segment blocks, each 16-byte aligned:
+//          ids   u32[F + 1] in REVERSE order: ids[p] sits at t2_off - 4 - 4p, and the slot
 //                of p = F holds PENDING -- the fast path needs no compare for "none"
-//          T2    u8[(Ks + 2) * (Ka + 1)]  at t2_off
-//          bitmap u32[nbw]
+//          T2    u8[(Ks + 2) * (Ka + 1)]  at t2_off (a multiple of 4)
+//          bitmap u32[nbw]  (further segments only)
 //          slow-path tables (SlowLayout below)
-//
-// Header words:
-//   w0 = float 2^-S          w1 = float -bmin
-//   w2 = t2_off / 16 | (Ka + 1) << 16 | nbw << 24
-//   w3 = acc_lo | cb << 16    acc_lo = multiple of 24 at or below the smallest accuracy,
-//                             cb = (bitmap_off - t2_off) / 4 + CB_BIAS - acc_lo / 24 (the bitmap
-//                             word for an accuracy a clamped to [acc_lo, acc_lo + 24 nbw - 1]
-//                             is word cb - CB_BIAS + a / 24 counted from t2_off)
 //
 // Per task in global memory (`regions`): keys u64[V] (pred_lat | acc_bp << 32, scan order,
 // F used; for Inactive entries the latency includes the loading latency) and ids u32[V], for
@@ -76,10 +72,8 @@ namespace infaas {
 constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
 constexpr uint32_t ACC_WORD_BITS = 24;
-constexpr uint32_t MAX_ACC_WORDS = 255;          // nbw is an 8-bit field: 6120 basis points
-constexpr uint32_t HDR_BYTES = 128;              // 8 copies x 16 bytes
-constexpr uint32_t IMAGE_T2_LIMIT = 1u << 20;    // t2_off / 16 is a 16-bit field
-constexpr uint32_t CB_BIAS = 512;                // keeps the header's bitmap field non-negative
+constexpr uint32_t MAX_ACC_WORDS = 420;          // accuracies 0 .. 10000 need at most 417 + 1 words
+constexpr uint32_t IMAGE_T2_LIMIT = 1u << 26;    // t2_off / 4 is a 24-bit field
 constexpr uint32_t SLO_CAP_FLOOR_US = (1u << 20) - 1u;  // the buckets cover latencies at least up to here
 constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-2)
 
@@ -88,13 +82,23 @@ constexpr uint32_t TASK_FLAG_NOT_INDEXED = 2u;   // list without index: the slow
 
 inline __host__ __device__ uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
-inline __host__ __device__ uint32_t image_rec_offset(uint32_t n_tasks) { return HDR_BYTES * (n_tasks + 1u); }
-inline __host__ __device__ uint32_t image_dummy_offset(uint32_t n_tasks) {
+inline __host__ __device__ uint32_t image_rec_offset(uint32_t n_tasks) { return round_up_u32(4u * (n_tasks + 1u), 128u); }
+inline __host__ __device__ uint32_t image_bitmap_offset(uint32_t n_tasks) {
   return image_rec_offset(n_tasks) + 4u * SLO_BUCKETS * (n_tasks + 1u);
 }
-inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks) { return image_dummy_offset(n_tasks) + 64u; }
+inline __host__ __device__ uint32_t image_dummy_offset(uint32_t n_tasks, uint32_t nbw) {
+  return round_up_u32(image_bitmap_offset(n_tasks) + 4u * nbw * (n_tasks + 1u), 64u);
+}
+inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks, uint32_t nbw) {
+  return image_dummy_offset(n_tasks, nbw) + 64u;
+}
+// The header word of a task without index (and of entry n_tasks): T2 is the one zero byte at
+// dummy + 16 with row width 0, the id slot of position 0 below it holds PENDING.
+inline __host__ __device__ uint32_t dummy_header(uint32_t n_tasks, uint32_t nbw) {
+  return (image_dummy_offset(n_tasks, nbw) + 16u) >> 2;
+}
 
-// Byte offsets of the slow-path tables inside a task's block, relative to their start
+// Byte offsets of the slow-path tables inside a segment's block, relative to their start
 // (8-byte aligned), for a list of F entries with Ks / Ka distinct latencies / accuracies.
 //   walk[o]   uint2 (pred_lat, acc | position << 16): the "stair" entries -- those no other
 //             entry beats in both latency and accuracy -- in ascending latency (Fs <= F of
@@ -119,22 +123,23 @@ inline __host__ __device__ SlowLayout slow_layout(uint32_t F, uint32_t Ks, uint3
   return L;
 }
 
-// Offsets inside a task's block and its size.
+// Offsets inside a segment's block and its size; `nbw` = 0 for a task's first segment (its
+// bitmap lives in the fixed part of the image).
 struct BlockLayout {
   uint32_t t2, bitmap, slow, bytes;   // ids start at 0; t2 = 4 (F + 1)
 };
 inline __host__ __device__ BlockLayout block_layout(uint32_t F, uint32_t Ks, uint32_t Ka, uint32_t nbw) {
   BlockLayout B;
-  B.t2 = round_up_u32(4u * (F + 1u), 16u);
+  B.t2 = 4u * (F + 1u);
   B.bitmap = round_up_u32(B.t2 + (Ks + 2u) * (Ka + 1u), 4u);
   B.slow = round_up_u32(B.bitmap + 4u * nbw, 8u);
-  B.bytes = round_up_u32(B.slow + slow_layout(F, Ks, Ka).bytes, 64u);
+  B.bytes = round_up_u32(B.slow + slow_layout(F, Ks, Ka).bytes, 16u);
   return B;
 }
-// Worst-case bytes of one task's block.
-inline __host__ __device__ uint32_t block_capacity(uint32_t V) {
+// Worst-case bytes of one segment's block.
+inline __host__ __device__ uint32_t block_capacity(uint32_t V, uint32_t nbw) {
   const uint32_t F = V < INDEX_MAX_F ? V : INDEX_MAX_F;
-  return block_layout(F, F, F, MAX_ACC_WORDS).bytes;
+  return block_layout(F, F, F, nbw).bytes;
 }
 inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_up_u32(14u * V, 64u); }
 
@@ -142,6 +147,8 @@ inline __host__ __device__ uint32_t region_capacity(uint32_t V) { return round_u
 // segment at index task, further segments at n_tasks + their index).
 //   x = image offset of the slow tables   y = F | Ks << 8 | Ka << 16   z = flags
 //   w = Fs | (1 + index of the task's next segment, 0 if none) << 8
+// Header of a further segment (xhdr, global memory):
+//   x = t2_off   y = Ka + 1   z = image offset of its bitmap   w = 0
 // ---------------------------------------------------------------------------------------
 // Device catalog.  "Slot" order: variants bucketed by task, ascending id inside a task;
 // task t owns slots task_off[t] .. task_off[t+1]-1 and all s_* arrays are indexed by slot.
@@ -174,7 +181,10 @@ struct DeviceCatalog {
 
   unsigned char *image;      // packed image, image_capacity bytes, 256-byte aligned
   uint32_t image_capacity;
-  uint32_t *image_hdr;       // [0]: bytes of the image (published by the rebuild kernel)
+  uint32_t *image_hdr;       // published by the rebuild kernel: [0] bytes of the image, [1] the bucket
+                             // scale 2^-S and [2] -bmin, both as float patterns
+  uint32_t acc_lo, nbw;      // accuracy window of every bitmap: acc_lo (multiple of 24) .. acc_lo + 24 nbw - 1
+  uint32_t lat_code_lo;      // bits(smallest profiled latency) >> 16: where the SLO buckets start
 
   unsigned long long *counters;  // [3] feasible, no-feasible, invalid
   unsigned long long *alloc_ctr; // rebuild kernel: block cursor (low 32 bits) | CTAs done allocating << 32;

@@ -85,11 +85,6 @@ struct SharedImage {
   __device__ __forceinline__ uint2 v2(uint32_t off) const {
     uint2 v; asm("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(base + off)); return v;
   }
-  __device__ __forceinline__ uint4 v4(uint32_t off) const {
-    uint4 v;
-    asm("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(base + off));
-    return v;
-  }
 };
 
 struct GlobalImage {
@@ -101,45 +96,61 @@ struct GlobalImage {
   __device__ __forceinline__ uint2 v2(uint32_t off) const {
     return __ldg(reinterpret_cast<const uint2 *>(base + off));
   }
-  __device__ __forceinline__ uint4 v4(uint32_t off) const {
-    return __ldg(reinterpret_cast<const uint4 *>(base + off));
-  }
 };
 
 // floor(a / 24) for a < 2^16 as the high half of a product (multiply pipe).
 __device__ __forceinline__ uint32_t div24(uint32_t a) { return __umulhi(a, 178956971u); }
 
-// k = #{distinct list accuracies < min_acc} from the bitmap with running popcounts.
-// w2, w3: header words (see common.cuh); t2: image offset of the task's T2.
+// What the lookups need that does not depend on the task: the bucket scale the last rebuild
+// used, the catalog's accuracy window, and where the fixed tables sit in the image.
+struct Fixed {
+  float scale, neg_bmin;      // bucket of an SLO: floor(bits(slo) * scale + neg_bmin), saturated to 0..255
+  uint32_t n_tasks;
+  uint32_t rec_off;           // image offset of the SLO records
+  uint32_t bm_off;            // image offset of the first tasks' bitmaps, less 4 * (acc_lo / 24)
+  uint32_t bm_stride;         // bytes of one bitmap
+  uint32_t acc_lo, acc_hi;    // accuracy window, both ends included
+};
+__device__ __forceinline__ Fixed make_fixed(const DeviceCatalog &c) {
+  Fixed f;
+  f.scale = __uint_as_float(c.image_hdr[1]);
+  f.neg_bmin = __uint_as_float(c.image_hdr[2]);
+  f.n_tasks = c.n_tasks;
+  f.rec_off = image_rec_offset(c.n_tasks);
+  f.bm_off = image_bitmap_offset(c.n_tasks) - 4u * (c.acc_lo / ACC_WORD_BITS);
+  f.bm_stride = 4u * c.nbw;
+  f.acc_lo = c.acc_lo;
+  f.acc_hi = c.acc_lo + ACC_WORD_BITS * c.nbw - 1u;
+  return f;
+}
+
+// k = #{distinct list accuracies < min_acc} from a bitmap with running popcounts whose word
+// for accuracy acc_lo sits at image offset bm0 + 4 * (acc_lo / 24).
 template <class Img>
-__device__ __forceinline__ uint32_t acc_rank(const Img &img, uint32_t w2, uint32_t w3, uint32_t t2,
-                                             uint32_t min_acc) {
-  const uint32_t acc_lo = w3 & 0xFFFFu, cb = __umulhi(w3, 1u << 16), nbw = __umulhi(w2, 1u << 8);
-  const uint32_t a = min(max(min_acc, acc_lo), acc_lo + ACC_WORD_BITS * nbw - 1u);
+__device__ __forceinline__ uint32_t acc_rank(const Img &img, const Fixed &fx, uint32_t bm0, uint32_t min_acc) {
+  const uint32_t a = min(max(min_acc, fx.acc_lo), fx.acc_hi);
   const uint32_t w = div24(a);
-  const uint32_t word = img.u32(t2 - 4u * CB_BIAS + ((cb + w) << 2));
+  const uint32_t word = img.u32(bm0 + (w << 2));
   const uint32_t below = word & ((1u << (a - w * ACC_WORD_BITS)) - 1u);   // prefix byte masked off: shift < 24
   return __umulhi(word, 1u << 8) + __popc(below);
 }
 
 // Fast path, straight-line: five loads, no compare.  Returns the variant id, or PENDING
 // when the tables cannot answer (nothing feasible, an SLO bucket with several latencies,
-// a task without index or out of range).  `hdr_lane` = 16 * (lane & 7): which of the 8
-// header copies this lane reads.
+// a task without index or out of range).
 template <class Img>
-__device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks, uint32_t rec_off,
-                                                uint32_t hdr_lane, uint32_t task, uint32_t slo,
+__device__ __forceinline__ uint32_t decide_fast(const Img &img, const Fixed &fx, uint32_t task, uint32_t slo,
                                                 uint32_t min_acc) {
-  const uint32_t t = min(task, n_tasks);
-  const uint4 h = img.v4(t * HDR_BYTES + hdr_lane);
+  const uint32_t t = min(task, fx.n_tasks);
+  const uint32_t h = img.u32(t << 2);
   // bucket of the SLO: floor(bits(slo) * 2^-S) - bmin, saturated to 0..255 by the conversion
   const float code = __uint2float_rz(__float_as_uint(__uint2float_rz(slo)));
   uint32_t j;
-  asm("cvt.rmi.sat.u8.f32 %0, %1;" : "=r"(j) : "f"(fmaf(code, __uint_as_float(h.x), __uint_as_float(h.y))));
-  const uint32_t rec = img.u32(rec_off + t * (4u * SLO_BUCKETS) + (j << 2));
+  asm("cvt.rmi.sat.u8.f32 %0, %1;" : "=r"(j) : "f"(fmaf(code, fx.scale, fx.neg_bmin)));
+  const uint32_t rec = img.u32(fx.rec_off + t * (4u * SLO_BUCKETS) + (j << 2));
   const uint32_t r = __umulhi(rec + (slo & 0x00FFFFFFu), 1u << 8);
-  const uint32_t t2 = (h.z & 0xFFFFu) << 4, width = (h.z >> 16) & 0xFFu;
-  const uint32_t k = acc_rank(img, h.z, h.w, t2, min_acc);
+  const uint32_t k = acc_rank(img, fx, fx.bm_off + t * fx.bm_stride, min_acc);
+  const uint32_t t2 = (h & 0x00FFFFFFu) << 2, width = h >> 24;
   const uint32_t pos = img.u8(t2 + r * width + k);
   return img.u32(t2 - 4u - (pos << 2));
 }
@@ -164,20 +175,19 @@ __device__ __forceinline__ uint32_t decide_fast(const Img &img, uint32_t n_tasks
 // segment's nearest miss into (best, best_id); a later segment wins only with a strictly
 // smaller distance, since its positions are all higher.
 template <class Img>
-__device__ __forceinline__ uint32_t slow_segment(const Img &img, const uint4 sl, const uint4 h, uint32_t slo,
-                                                 uint32_t min_acc, unsigned long long &best,
-                                                 uint32_t &best_id) {
+__device__ __forceinline__ uint32_t slow_segment(const Img &img, const Fixed &fx, const uint4 sl, uint32_t t2,
+                                                 uint32_t width, uint32_t bm0, uint32_t slo, uint32_t min_acc,
+                                                 unsigned long long &best, uint32_t &best_id) {
   const uint32_t F = sl.y & 0xFFu, Ks = (sl.y >> 8) & 0xFFu, Ka = sl.y >> 16, Fs = sl.w & 0xFFu;
   const SlowLayout SL = slow_layout(F, Ks, Ka);
   const uint32_t so = sl.x;
-  const uint32_t t2 = (h.z & 0xFFFFu) << 4, width = (h.z >> 16) & 0xFFu;
   uint32_t r = 0;                                            // r = #{Pd <= slo}
 #pragma unroll
   for (uint32_t step = 128; step; step >>= 1) {
     const uint32_t probe = r + step;
     if (probe <= Ks && img.u32(so + SL.Pd + ((probe - 1u) << 2)) <= slo) r = probe;
   }
-  const uint32_t k = acc_rank(img, h.z, h.w, t2, min_acc);
+  const uint32_t k = acc_rank(img, fx, bm0, min_acc);
   const uint32_t pos = img.u8(t2 + r * width + k);
   if (pos < F) return img.u32(t2 - 4u - (pos << 2));
   unsigned long long mine = ~0ull;        // this segment's nearest miss
@@ -218,7 +228,7 @@ __device__ __forceinline__ uint32_t slow_segment(const Img &img, const uint4 sl,
 }
 
 template <class Img>
-__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, uint32_t task,
+__device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCatalog &c, const Fixed &fx, uint32_t task,
                                                 uint32_t slo, uint32_t min_acc) {
   if (task >= c.n_tasks) return INFAAS_INVALID;
   uint4 sl = __ldg(c.slow + task);
@@ -226,16 +236,18 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
   unsigned long long best = ~0ull;
   uint32_t best_p = 0;
   if (!(sl.z & TASK_FLAG_NOT_INDEXED)) {
-    // the list's segments in order: the first has its header in the image, the others
-    // (lists longer than INDEX_MAX_F) in global memory
-    uint4 h = img.v4(task * HDR_BYTES + ((threadIdx.x & 7u) << 4));   // this lane's copy
+    // the list's segments in order: the first has its header word and bitmap in the fixed part
+    // of the image, the others (lists longer than INDEX_MAX_F) a header in global memory
+    const uint32_t h = img.u32(task << 2);
+    uint32_t t2 = (h & 0x00FFFFFFu) << 2, width = h >> 24, bm0 = fx.bm_off + task * fx.bm_stride;
     for (;;) {
-      const uint32_t d = slow_segment(img, sl, h, slo, min_acc, best, best_p);
+      const uint32_t d = slow_segment(img, fx, sl, t2, width, bm0, slo, min_acc, best, best_p);
       if (d != PENDING) return d;
       const uint32_t next = sl.w >> 8;                       // 1 + index of the next segment
       if (next == 0u) break;
       sl = __ldg(c.slow + c.n_tasks + next - 1u);
-      h = __ldg(c.xhdr + next - 1u);
+      const uint4 xh = __ldg(c.xhdr + next - 1u);
+      t2 = xh.x; width = xh.y; bm0 = xh.z - 4u * (fx.acc_lo / ACC_WORD_BITS);
     }
     return INFAAS_NO_FEASIBLE | best_p;
   }
@@ -274,12 +286,12 @@ struct Park {
 
 // Resolve the 32 parked queries [first, first + count), one per lane.
 template <class Img>
-__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, uint32_t *out,
+__device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, const Fixed &fx, uint32_t *out,
                                                const Park &pk, uint32_t first, uint32_t count) {
   const uint32_t lane = threadIdx.x & 31;
   if (lane < count) {
     const uint32_t ta = pk.ta[first + lane];
-    out[pk.rel[first + lane]] = decide_slow(img, c, ta & 0xFFFFu, pk.slo[first + lane], ta >> 16);
+    out[pk.rel[first + lane]] = decide_slow(img, c, fx, ta & 0xFFFFu, pk.slo[first + lane], ta >> 16);
   }
 }
 
@@ -287,7 +299,7 @@ __device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatal
 // queries, data in ta[i] / s[i], offset rel + i); flush whenever 32 are waiting.  All
 // lanes of the warp call this together.
 template <class Img>
-__device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatalog &c, uint32_t *out, Park &pk,
+__device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatalog &c, const Fixed &fx, uint32_t *out, Park &pk,
                                                uint32_t pm, uint32_t rel, const uint32_t (&ta)[4],
                                                const uint32_t (&s)[4]) {
   const uint32_t lane_lt = (1u << (threadIdx.x & 31)) - 1u;
@@ -304,7 +316,7 @@ __device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatal
     __syncwarp();
     if (pk.cnt >= 32) {
       pk.cnt -= 32;
-      resolve_parked(img, c, out, pk, pk.cnt, 32);
+      resolve_parked(img, c, fx, out, pk, pk.cnt, 32);
       __syncwarp();
     }
   }
@@ -314,10 +326,8 @@ template <class Img>
 __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
                                             uint64_t q0, uint32_t span, uint32_t *park_all, uint2 t4, uint4 s4,
                                             uint2 a4) {
-  const uint32_t n_tasks = c.n_tasks;
-  const uint32_t rec_off = image_rec_offset(n_tasks);
+  const Fixed fx = make_fixed(c);
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t hdr_lane = (lane & 7u) << 4;
   Park pk;
   pk.rel = park_all + warp * (3 * PARK_CAP);
   pk.ta = pk.rel + PARK_CAP;
@@ -344,10 +354,10 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
     const uint32_t aq[4] = {a.x & 0xFFFFu, a.x >> 16, a.y & 0xFFFFu, a.y >> 16};
     const uint32_t sq[4] = {s.x, s.y, s.z, s.w};
     uint4 d;
-    d.x = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[0], sq[0], aq[0]);
-    d.y = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[1], sq[1], aq[1]);
-    d.z = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[2], sq[2], aq[2]);
-    d.w = decide_fast(img, n_tasks, rec_off, hdr_lane, tq[3], sq[3], aq[3]);
+    d.x = decide_fast(img, fx, tq[0], sq[0], aq[0]);
+    d.y = decide_fast(img, fx, tq[1], sq[1], aq[1]);
+    d.z = decide_fast(img, fx, tq[2], sq[2], aq[2]);
+    d.w = decide_fast(img, fx, tq[3], sq[3], aq[3]);
     const uint32_t rel = tile * WARP_TILE + lane * 4u;
     // PENDING slots are overwritten by the lane that resolves them, after a warp barrier
     __stcs(reinterpret_cast<uint4 *>(out + rel), d);
@@ -357,7 +367,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
       const uint32_t ta[4] = {tq[0] | (aq[0] << 16), tq[1] | (aq[1] << 16), tq[2] | (aq[2] << 16),
                               tq[3] | (aq[3] << 16)};
       __syncwarp();
-      park_and_flush(img, c, out, pk, pm, rel, ta, sq);
+      park_and_flush(img, c, fx, out, pk, pm, rel, ta, sq);
     }
   }
   // ragged tail of the CTA's range (fewer than WARP_TILE queries): one warp, scalar accesses
@@ -372,15 +382,15 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
         sq[0] = q.slo[i];
         slo_or |= sq[0];
         ta[0] = tk | (ac << 16);
-        d = decide_fast(img, n_tasks, rec_off, hdr_lane, tk, sq[0], ac);
+        d = decide_fast(img, fx, tk, sq[0], ac);
         out[rel] = d;
       }
       __syncwarp();
-      park_and_flush(img, c, out, pk, d >> 31, rel, ta, sq);
+      park_and_flush(img, c, fx, out, pk, d >> 31, rel, ta, sq);
     }
   }
   __syncwarp();
-  resolve_parked(img, c, out, pk, 0, pk.cnt);
+  resolve_parked(img, c, fx, out, pk, 0, pk.cnt);
   slo_or = __reduce_or_sync(0xFFFFFFFFu, slo_or);
   if (lane == 0 && (slo_or & ~*c.slo_seen)) atomicOr(c.slo_seen, slo_or);
 }

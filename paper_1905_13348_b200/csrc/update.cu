@@ -189,7 +189,7 @@ struct IndexScratch {          // shared memory used while building one task's i
   uint16_t acc[256], Ad[256];
   unsigned char idxP[256], idxA[256], firstP[256], firstA[256], on_stair[256];
   uint32_t bcnt[256], bthr[256];    // per SLO bucket: distinct latencies inside it, one of them
-  uint32_t wbits[256];              // per bitmap word: the accuracies present
+  uint32_t wbits[MAX_ACC_WORDS];    // per bitmap word: the accuracies present
   unsigned long long Lmask[4][256], Amask[4][256];   // [word][rank]: positions by latency rank < r / accuracy rank >= k
   // per latency rank: the most accurate entry (acc << 16 | 0xFFFF - position, 0 = none) and
   // 1 + position of its stair entry (0 = none); per accuracy rank: the fastest entry
@@ -251,15 +251,29 @@ __device__ __forceinline__ void warp_prefix_count(const uint16_t *in, unsigned c
   }
 }
 
-// Header of a task without index (also entry n_tasks): every query reads "none".
-__device__ __forceinline__ uint4 dummy_header(uint32_t n_tasks) {
-  const uint32_t dummy = image_dummy_offset(n_tasks);
-  // T2 (one byte, 0) at dummy + 16, the id slot of position 0 (PENDING) just below it, the bitmap
-  // (one word, 0) at dummy + 32
-  return make_uint4(0u, 0u, ((dummy + 16u) >> 4) | (0u << 16) | (1u << 24), 0u | ((4u + CB_BIAS) << 16));
+// Fixed part of the image for a task without index (also entry n_tasks): a header word,
+// records and a bitmap that make every query of the task read "none".  All threads.
+__device__ __forceinline__ void write_dummy_task(const DeviceCatalog &c, uint32_t t) {
+  const uint32_t T = c.n_tasks;
+  if (threadIdx.x == 0) reinterpret_cast<uint32_t *>(c.image)[t] = dummy_header(T, c.nbw);
+  uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T)) + t * SLO_BUCKETS;
+  for (uint32_t j = threadIdx.x; j < SLO_BUCKETS; j += blockDim.x) rec[j] = 0u;
+  uint32_t *bm = reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(T)) + t * c.nbw;
+  for (uint32_t j = threadIdx.x; j < c.nbw; j += blockDim.x) bm[j] = 0u;
 }
-__device__ __forceinline__ void write_header(const DeviceCatalog &c, uint32_t t, uint4 h) {
-  if (threadIdx.x < HDR_BYTES / 16u) reinterpret_cast<uint4 *>(c.image + HDR_BYTES * t)[threadIdx.x] = h;
+
+// Bucket scale of the SLO records: S (16..23) and bmin such that SLO_BUCKETS - 1 buckets of
+// 2^S float patterns cover everything from the catalog's smallest profiled latency up to the
+// largest SLO asked for so far (as a bit mask: every SLO seen is <= cap).
+__device__ __forceinline__ void bucket_scale(const DeviceCatalog &c, uint32_t &Sh, uint32_t &bmin) {
+  uint32_t cap = *c.slo_seen | SLO_CAP_FLOOR_US;
+  cap |= cap >> 1; cap |= cap >> 2; cap |= cap >> 4; cap |= cap >> 8; cap |= cap >> 16;
+  const uint32_t clo = c.lat_code_lo;
+  const uint32_t chi = max(clo, __float_as_uint(__uint2float_rz(cap)) >> 16);
+  uint32_t sh = 0;
+  while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
+  bmin = clo >> sh;
+  Sh = 16u + sh;
 }
 
 // Sum / OR over the aligned group of 8 lanes this lane belongs to.
@@ -288,7 +302,7 @@ __device__ __forceinline__ unsigned long long place_block_issue(const DeviceCata
 __device__ __forceinline__ uint32_t place_block_finish(const DeviceCatalog &c, unsigned long long old,
                                                        uint32_t bytes, bool done) {
   if (done && (uint32_t)(old >> 32) == gridDim.x - 1u) {
-    c.image_hdr[0] = image_var_offset(c.n_tasks) + (uint32_t)old + bytes;
+    c.image_hdr[0] = image_var_offset(c.n_tasks, c.nbw) + (uint32_t)old + bytes;
     *c.alloc_ctr = 0ull;
   }
   return (uint32_t)old;
@@ -296,13 +310,12 @@ __device__ __forceinline__ uint32_t place_block_finish(const DeviceCatalog &c, u
 
 // Builds the exact index of a list of F <= INDEX_MAX_F entries (layout in common.cuh) into
 // a block of the image obtained from the block cursor.  S.pred / S.acc / S.ids hold the
-// list in scan order.  Returns false (all threads) if the list cannot be indexed: its
-// accuracies span more than the bitmap supports, or the block lies beyond what the 16-bit
-// offsets address.  blockDim = REBUILD_THREADS: the pair loops give every entry 8 lanes, and
+// list in scan order.  Returns false (all threads) if the list cannot be indexed: its block
+// lies beyond the image's capacity or beyond what the header's offset field addresses.  blockDim = REBUILD_THREADS: the pair loops give every entry 8 lanes, and
 // the tables, which do not depend on each other, are written by different groups of warps.
-// `xi`: 0xFFFFFFFF for the task's first segment (header and SLO records go into the image), else
-// the index of this further segment (header to xhdr[xi], no records: only the slow path comes
-// here).  `next`: 1 + index of the task's next segment, 0 if this is the last (the CTA's last
+// `xi`: 0xFFFFFFFF for the task's first segment (header word, SLO records and bitmap go into the
+// fixed part of the image), else the index of this further segment (header to xhdr[xi], bitmap
+// into the block, no records: only the slow path comes here).  `next`: 1 + index of the task's next segment, 0 if this is the last (the CTA's last
 // allocation, then).
 __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, IndexScratch &S, uint32_t xi,
                             uint32_t next) {
@@ -330,7 +343,8 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     if (p < F && sub == 0) { S.firstP[p] = !(dup & 1u); S.firstA[p] = !(dup & 2u); S.on_stair[p] = !(dup & 4u); }
   }
   if (tid == 0) { S.ks = 0; S.ka = 0; S.fs = 0; }
-  if (tid < 256) { S.rankA[tid] = 0u; S.rankB[tid] = ~0ull; S.stair_at[tid] = 0; S.bcnt[tid] = 0u; S.wbits[tid] = 0u; }
+  if (tid < 256) { S.rankA[tid] = 0u; S.rankB[tid] = ~0ull; S.stair_at[tid] = 0; S.bcnt[tid] = 0u; }
+  if (tid < MAX_ACC_WORDS) S.wbits[tid] = 0u;
   __syncthreads();
   // ... and their ranks
   for (uint32_t p0 = 0; p0 < F; p0 += PB) {
@@ -366,23 +380,15 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   if ((tid >> 5) == 2) warp_prefix_count(S.stair_at, S.ord_start, Ks);
   // block layout and its place in the image; the atomic that places it is in flight while the
   // masks below are built
-  const uint32_t acc_lo = (S.Ad[0] / ACC_WORD_BITS) * ACC_WORD_BITS;
-  const uint32_t nbw = (S.Ad[Ka - 1] + 1u - acc_lo) / ACC_WORD_BITS + 1u;
+  const uint32_t acc_lo = c.acc_lo, nbw = c.nbw;      // the catalog's accuracy window
   const uint32_t width = Ka + 1u;
-  const BlockLayout BL = block_layout(F, Ks, Ka, nbw);
+  const BlockLayout BL = block_layout(F, Ks, Ka, first ? 0u : nbw);
   const SlowLayout SL = slow_layout(F, Ks, Ka);
-  const bool fits = nbw <= MAX_ACC_WORDS;
   unsigned long long placed = 0;
-  if (tid == 0) placed = place_block_issue(c, fits ? BL.bytes : 0u, next == 0u);
-  // SLO buckets: they cover the list's latencies up to the largest SLO asked for so far (as a
-  // bit mask: every SLO seen is <= cap); larger latencies share bucket 255
-  uint32_t cap = *c.slo_seen | SLO_CAP_FLOOR_US;
-  cap |= cap >> 1; cap |= cap >> 2; cap |= cap >> 4; cap |= cap >> 8; cap |= cap >> 16;
-  const uint32_t clo = float_bits(S.Pd[0]) >> 16;
-  const uint32_t chi = max(clo, float_bits(min(S.Pd[Ks - 1], cap)) >> 16);
-  uint32_t sh = 0;
-  while ((chi >> sh) - (clo >> sh) > SLO_BUCKETS - 2) ++sh;
-  const uint32_t bmin = clo >> sh, Sh = 16u + sh;
+  if (tid == 0) placed = place_block_issue(c, BL.bytes, next == 0u);
+  // SLO buckets: larger latencies than the largest SLO asked for so far share bucket 255
+  uint32_t bmin, Sh;
+  bucket_scale(c, Sh, bmin);
   for (uint32_t i = tid; i < Ks; i += B) {
     const uint32_t b = min(max(float_bits(S.Pd[i]) >> Sh, bmin) - bmin, SLO_BUCKETS - 1);
     atomicAdd(&S.bcnt[b], 1u);
@@ -408,8 +414,8 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   }
 
   if (tid == 0) {
-    uint32_t base = image_var_offset(c.n_tasks) + place_block_finish(c, placed, fits ? BL.bytes : 0u, next == 0u);
-    if (!fits || base + BL.bytes > c.image_capacity || base + BL.t2 >= IMAGE_T2_LIMIT) base = 0xFFFFFFFFu;
+    uint32_t base = image_var_offset(c.n_tasks, nbw) + place_block_finish(c, placed, BL.bytes, next == 0u);
+    if (base + BL.bytes > c.image_capacity || base + BL.t2 >= IMAGE_T2_LIMIT) base = 0xFFFFFFFFu;
     S.base = base;
   }
   __syncthreads();
@@ -454,8 +460,10 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     rec[j] = r;
   }
 
-  // accuracy bitmap with running popcounts: warps 24-27, 128 words a round, same scheme
-  uint32_t *bitmap = reinterpret_cast<uint32_t *>(blk + BL.bitmap);
+  // accuracy bitmap with running popcounts: warps 24-27, 128 words a round, same scheme; a
+  // first segment's bitmap goes into the fixed part of the image
+  uint32_t *bitmap = first ? reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(c.n_tasks)) + t * nbw
+                           : reinterpret_cast<uint32_t *>(blk + BL.bitmap);
   if (tid >= 3 * B / 4 && tid < 3 * B / 4 + 128u) {
     const uint32_t lane = tid & 31u;
     for (uint32_t w0 = 0; w0 < nbw; w0 += 128u) {              // uniform over the four warps
@@ -512,13 +520,11 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
     T2[cell] = (unsigned char)pos;
   });
 
-  const uint32_t cb = ((BL.bitmap - BL.t2) >> 2) + CB_BIAS - acc_lo / ACC_WORD_BITS;
-  const uint4 hdr = make_uint4((127u - Sh) << 23, __float_as_uint(-(float)bmin),
-                               ((base + BL.t2) >> 4) | (width << 16) | (nbw << 24), acc_lo | (cb << 16));
-  if (first) write_header(c, t, hdr);
-  else if (tid == 0) c.xhdr[xi] = hdr;
-  if (tid == 0)
+  if (tid == 0) {
+    if (first) reinterpret_cast<uint32_t *>(c.image)[t] = ((base + BL.t2) >> 2) | (width << 24);
+    else c.xhdr[xi] = make_uint4(base + BL.t2, width, base + BL.bitmap, 0u);
     c.slow[first ? t : c.n_tasks + xi] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs | (next << 8));
+  }
   return true;
 }
 
@@ -816,19 +822,22 @@ rebuild_kernel(DeviceCatalog c, int advance, uint32_t window_us) {
   }
   if (!counted && tid == 0) place_block_finish(c, place_block_issue(c, 0u, true), 0u, true);   // nothing (more) to place
   if (!indexed) {
-    // no index: header and records that make every query of this task read "none"
-    write_header(c, t, dummy_header(c.n_tasks));
-    uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
-    for (uint32_t j = tid; j < SLO_BUCKETS; j += B) rec[j] = 0u;
+    // no index: every query of this task reads "none"
+    write_dummy_task(c, t);
     if (tid == 0) c.slow[t] = make_uint4(0u, 0u, F == 0 ? TASK_FLAG_INVALID : TASK_FLAG_NOT_INDEXED, 0u);
   }
   if (t == 0) {
-    // entry n_tasks (queries whose task is out of range) and the dummy block
-    const uint32_t T = c.n_tasks, dummy = image_dummy_offset(T);
-    write_header(c, T, dummy_header(T));
-    uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T)) + T * SLO_BUCKETS;
-    for (uint32_t j = tid; j < SLO_BUCKETS; j += B) rec[j] = 0u;
+    // entry n_tasks (queries whose task is out of range), the dummy block, and the bucket scale
+    // every CTA has used, for the selection kernel
+    const uint32_t T = c.n_tasks, dummy = image_dummy_offset(T, c.nbw);
+    write_dummy_task(c, T);
     if (tid < 16) reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid == 3 ? PENDING : 0u;
+    if (tid == 0) {
+      uint32_t Sh, bmin;
+      bucket_scale(c, Sh, bmin);
+      c.image_hdr[1] = (127u - Sh) << 23;
+      c.image_hdr[2] = __float_as_uint(-(float)bmin);
+    }
   }
   if (tid == 0) c.f_len[t] = F;
 }
