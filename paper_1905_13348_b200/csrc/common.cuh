@@ -51,10 +51,11 @@ namespace infaas {
 // and nbw words), so the word an accuracy falls into does not depend on the task.
 //
 // Image (what the selection kernel stages in shared memory):
-//   hdr    (n_tasks + 1) u32, one per task: t2_off / 4 | (Ka + 1) << 24; entry n_tasks serves
+//   hdr    (n_tasks + 1) u32, one per task: t2_off | (Ka + 1) << 24; entry n_tasks serves
 //          queries whose task is out of range; padded to 128 bytes
-//   rec    (n_tasks + 1) x SLO_BUCKETS u32 records
-//   bitmap (n_tasks + 1) x nbw u32: the accuracy bitmaps of the tasks' first segments
+//   rec    (n_tasks + 1) x SLO_BUCKETS u32 records, REC_STRIDE bytes apart
+//   bitmap (n_tasks + 1) x nbw u32: the accuracy bitmaps of the tasks' first segments,
+//          bitmap_stride(nbw) bytes apart
 //   dummy  64 bytes (what tasks without an index point at: every query of theirs reads
 //          "none" and goes to the slow path)
 //   var    per-segment blocks, each 16-byte aligned:
@@ -73,7 +74,7 @@ constexpr uint32_t INDEX_MAX_F = 248;
 constexpr uint32_t SLO_BUCKETS = 256;
 constexpr uint32_t ACC_WORD_BITS = 24;
 constexpr uint32_t MAX_ACC_WORDS = 420;          // accuracies 0 .. 10000 need at most 417 + 1 words
-constexpr uint32_t IMAGE_T2_LIMIT = 1u << 26;    // t2_off / 4 is a 24-bit field
+constexpr uint32_t IMAGE_T2_LIMIT = 1u << 24;    // t2_off is a 24-bit field
 constexpr uint32_t SLO_CAP_FLOOR_US = (1u << 20) - 1u;  // the buckets cover latencies at least up to here
 constexpr uint32_t PENDING = 0xFFFFFFFEu;        // never a valid decision (ids stop at 2^31-2)
 
@@ -82,12 +83,17 @@ constexpr uint32_t TASK_FLAG_NOT_INDEXED = 2u;   // list without index: the slow
 
 inline __host__ __device__ uint32_t round_up_u32(uint32_t x, uint32_t a) { return (x + a - 1) / a * a; }
 
+// A task's records and its bitmap start an odd number of words after the previous task's, so
+// that the tasks' hot entries (the same buckets, the lowest bitmap word) fall into different
+// shared-memory banks.
+constexpr uint32_t REC_STRIDE = 4u * (SLO_BUCKETS + 1u);   // bytes from one task's records to the next's
+inline __host__ __device__ uint32_t bitmap_stride(uint32_t nbw) { return 4u * (nbw | 1u); }   // same, bitmaps
 inline __host__ __device__ uint32_t image_rec_offset(uint32_t n_tasks) { return round_up_u32(4u * (n_tasks + 1u), 128u); }
 inline __host__ __device__ uint32_t image_bitmap_offset(uint32_t n_tasks) {
-  return image_rec_offset(n_tasks) + 4u * SLO_BUCKETS * (n_tasks + 1u);
+  return image_rec_offset(n_tasks) + REC_STRIDE * (n_tasks + 1u);
 }
 inline __host__ __device__ uint32_t image_dummy_offset(uint32_t n_tasks, uint32_t nbw) {
-  return round_up_u32(image_bitmap_offset(n_tasks) + 4u * nbw * (n_tasks + 1u), 64u);
+  return round_up_u32(image_bitmap_offset(n_tasks) + bitmap_stride(nbw) * (n_tasks + 1u), 64u);
 }
 inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks, uint32_t nbw) {
   return image_dummy_offset(n_tasks, nbw) + 64u;
@@ -95,7 +101,7 @@ inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks, uint32_t 
 // The header word of a task without index (and of entry n_tasks): T2 is the one zero byte at
 // dummy + 16 with row width 0, the id slot of position 0 below it holds PENDING.
 inline __host__ __device__ uint32_t dummy_header(uint32_t n_tasks, uint32_t nbw) {
-  return (image_dummy_offset(n_tasks, nbw) + 16u) >> 2;
+  return image_dummy_offset(n_tasks, nbw) + 16u;
 }
 
 // Byte offsets of the slow-path tables inside a segment's block, relative to their start

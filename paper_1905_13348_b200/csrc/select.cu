@@ -25,7 +25,7 @@ constexpr int SELECT_THREADS = 1024;
 constexpr int SELECT_WARPS = SELECT_THREADS / 32;
 constexpr uint32_t WARP_TILE = 128;              // queries per warp and iteration
 constexpr uint32_t PARK_CAP = 64;                // parked queries per warp (flushed at 32)
-constexpr uint32_t PARK_BYTES = SELECT_WARPS * PARK_CAP * 12;
+constexpr uint32_t PARK_BYTES = SELECT_WARPS * PARK_CAP * 16;
 constexpr uint32_t STAGE_CHUNK = 32768;          // bytes per bulk copy
 constexpr uint32_t STAGE_POLL_LIMIT = 1u << 22;  // bounded wait on the staging barrier
 constexpr uint32_t MAX_SPAN = 1u << 31;          // queries per CTA (offsets are 32-bit)
@@ -118,7 +118,7 @@ __device__ __forceinline__ Fixed make_fixed(const DeviceCatalog &c) {
   f.n_tasks = c.n_tasks;
   f.rec_off = image_rec_offset(c.n_tasks);
   f.bm_off = image_bitmap_offset(c.n_tasks) - 4u * (c.acc_lo / ACC_WORD_BITS);
-  f.bm_stride = 4u * c.nbw;
+  f.bm_stride = bitmap_stride(c.nbw);
   f.acc_lo = c.acc_lo;
   f.acc_hi = c.acc_lo + ACC_WORD_BITS * c.nbw - 1u;
   return f;
@@ -126,9 +126,9 @@ __device__ __forceinline__ Fixed make_fixed(const DeviceCatalog &c) {
 
 // k = #{distinct list accuracies < min_acc} from a bitmap with running popcounts whose word
 // for accuracy acc_lo sits at image offset bm0 + 4 * (acc_lo / 24).
-template <class Img>
+template <bool Clamped, class Img>
 __device__ __forceinline__ uint32_t acc_rank(const Img &img, const Fixed &fx, uint32_t bm0, uint32_t min_acc) {
-  const uint32_t a = min(max(min_acc, fx.acc_lo), fx.acc_hi);
+  const uint32_t a = Clamped ? min_acc : min(max(min_acc, fx.acc_lo), fx.acc_hi);
   const uint32_t w = div24(a);
   const uint32_t word = img.u32(bm0 + (w << 2));
   const uint32_t below = word & ((1u << (a - w * ACC_WORD_BITS)) - 1u);   // prefix byte masked off: shift < 24
@@ -138,19 +138,20 @@ __device__ __forceinline__ uint32_t acc_rank(const Img &img, const Fixed &fx, ui
 // Fast path, straight-line: five loads, no compare.  Returns the variant id, or PENDING
 // when the tables cannot answer (nothing feasible, an SLO bucket with several latencies,
 // a task without index or out of range).
-template <class Img>
+// `Clamped`: the caller has already limited the task to n_tasks and the accuracy to the window.
+template <bool Clamped, class Img>
 __device__ __forceinline__ uint32_t decide_fast(const Img &img, const Fixed &fx, uint32_t task, uint32_t slo,
                                                 uint32_t min_acc) {
-  const uint32_t t = min(task, fx.n_tasks);
+  const uint32_t t = Clamped ? task : min(task, fx.n_tasks);
   const uint32_t h = img.u32(t << 2);
   // bucket of the SLO: floor(bits(slo) * 2^-S) - bmin, saturated to 0..255 by the conversion
   const float code = __uint2float_rz(__float_as_uint(__uint2float_rz(slo)));
   uint32_t j;
   asm("cvt.rmi.sat.u8.f32 %0, %1;" : "=r"(j) : "f"(fmaf(code, fx.scale, fx.neg_bmin)));
-  const uint32_t rec = img.u32(fx.rec_off + t * (4u * SLO_BUCKETS) + (j << 2));
+  const uint32_t rec = img.u32(fx.rec_off + t * REC_STRIDE + (j << 2));
   const uint32_t r = __umulhi(rec + (slo & 0x00FFFFFFu), 1u << 8);
-  const uint32_t k = acc_rank(img, fx, fx.bm_off + t * fx.bm_stride, min_acc);
-  const uint32_t t2 = (h & 0x00FFFFFFu) << 2, width = h >> 24;
+  const uint32_t k = acc_rank<Clamped>(img, fx, fx.bm_off + t * fx.bm_stride, min_acc);
+  const uint32_t t2 = h & 0x00FFFFFFu, width = h >> 24;
   const uint32_t pos = img.u8(t2 + r * width + k);
   return img.u32(t2 - 4u - (pos << 2));
 }
@@ -187,7 +188,7 @@ __device__ __forceinline__ uint32_t slow_segment(const Img &img, const Fixed &fx
     const uint32_t probe = r + step;
     if (probe <= Ks && img.u32(so + SL.Pd + ((probe - 1u) << 2)) <= slo) r = probe;
   }
-  const uint32_t k = acc_rank(img, fx, bm0, min_acc);
+  const uint32_t k = acc_rank<false>(img, fx, bm0, min_acc);
   const uint32_t pos = img.u8(t2 + r * width + k);
   if (pos < F) return img.u32(t2 - 4u - (pos << 2));
   unsigned long long mine = ~0ull;        // this segment's nearest miss
@@ -239,7 +240,7 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
     // the list's segments in order: the first has its header word and bitmap in the fixed part
     // of the image, the others (lists longer than INDEX_MAX_F) a header in global memory
     const uint32_t h = img.u32(task << 2);
-    uint32_t t2 = (h & 0x00FFFFFFu) << 2, width = h >> 24, bm0 = fx.bm_off + task * fx.bm_stride;
+    uint32_t t2 = h & 0x00FFFFFFu, width = h >> 24, bm0 = fx.bm_off + task * fx.bm_stride;
     for (;;) {
       const uint32_t d = slow_segment(img, fx, sl, t2, width, bm0, slo, min_acc, best, best_p);
       if (d != PENDING) return d;
@@ -277,10 +278,10 @@ struct Queries {
   uint32_t *__restrict__ decision;
 };
 
-// A warp's park list in shared memory: offset of the query from the CTA's first query,
-// task | min_acc << 16, and SLO.
+// A warp's park list in shared memory, one 16-byte entry per parked query: offset of the
+// query from the CTA's first query, SLO, task | min_acc << 16, and a spare word.
 struct Park {
-  uint32_t *rel, *ta, *slo;
+  uint4 *e;
   uint32_t cnt;
 };
 
@@ -290,8 +291,8 @@ __device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatal
                                                const Park &pk, uint32_t first, uint32_t count) {
   const uint32_t lane = threadIdx.x & 31;
   if (lane < count) {
-    const uint32_t ta = pk.ta[first + lane];
-    out[pk.rel[first + lane]] = decide_slow(img, c, fx, ta & 0xFFFFu, pk.slo[first + lane], ta >> 16);
+    const uint4 e = pk.e[first + lane];
+    out[e.x] = decide_slow(img, c, fx, e.z & 0xFFFFu, e.y, e.z >> 16);
   }
 }
 
@@ -306,10 +307,10 @@ __device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatal
   unsigned m;
   while ((m = __ballot_sync(0xFFFFFFFFu, pm != 0u)) != 0u) {
     if (pm) {
-      const uint32_t i = __ffs(pm) - 1u, slot = pk.cnt + __popc(m & lane_lt);
-      pk.rel[slot] = rel + i;
-      pk.ta[slot] = i == 0 ? ta[0] : i == 1 ? ta[1] : i == 2 ? ta[2] : ta[3];
-      pk.slo[slot] = i == 0 ? s[0] : i == 1 ? s[1] : i == 2 ? s[2] : s[3];
+      const uint32_t i = __ffs(pm) - 1u;
+      pk.e[pk.cnt + __popc(m & lane_lt)] =
+          make_uint4(rel + i, i == 0 ? s[0] : i == 1 ? s[1] : i == 2 ? s[2] : s[3],
+                     i == 0 ? ta[0] : i == 1 ? ta[1] : i == 2 ? ta[2] : ta[3], 0u);
       pm &= pm - 1u;
     }
     pk.cnt += __popc(m);
@@ -324,17 +325,16 @@ __device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatal
 
 template <class Img>
 __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
-                                            uint64_t q0, uint32_t span, uint32_t *park_all, uint2 t4, uint4 s4,
+                                            uint64_t q0, uint32_t span, uint4 *park_all, uint2 t4, uint4 s4,
                                             uint2 a4) {
   const Fixed fx = make_fixed(c);
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Park pk;
-  pk.rel = park_all + warp * (3 * PARK_CAP);
-  pk.ta = pk.rel + PARK_CAP;
-  pk.slo = pk.ta + PARK_CAP;
+  pk.e = park_all + warp * PARK_CAP;
   pk.cnt = 0;
   uint32_t *out = q.decision + q0;
   const uint32_t full_tiles = span / WARP_TILE;
+  const uint32_t t_max2 = fx.n_tasks * 0x10001u, a_lo2 = fx.acc_lo * 0x10001u, a_hi2 = fx.acc_hi * 0x10001u;
 
   // full tiles: 4 consecutive queries per lane, 128-bit loads, next tile prefetched (the
   // first tile was loaded by the caller while the image was being staged)
@@ -353,11 +353,15 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
     const uint32_t tq[4] = {t.x & 0xFFFFu, t.x >> 16, t.y & 0xFFFFu, t.y >> 16};
     const uint32_t aq[4] = {a.x & 0xFFFFu, a.x >> 16, a.y & 0xFFFFu, a.y >> 16};
     const uint32_t sq[4] = {s.x, s.y, s.z, s.w};
+    // tasks limited to n_tasks (the entry of "out of range") and accuracies to the bitmaps'
+    // window, two 16-bit values per instruction
+    const uint32_t tcx = __vminu2(t.x, t_max2), tcy = __vminu2(t.y, t_max2);
+    const uint32_t acx = __vminu2(__vmaxu2(a.x, a_lo2), a_hi2), acy = __vminu2(__vmaxu2(a.y, a_lo2), a_hi2);
     uint4 d;
-    d.x = decide_fast(img, fx, tq[0], sq[0], aq[0]);
-    d.y = decide_fast(img, fx, tq[1], sq[1], aq[1]);
-    d.z = decide_fast(img, fx, tq[2], sq[2], aq[2]);
-    d.w = decide_fast(img, fx, tq[3], sq[3], aq[3]);
+    d.x = decide_fast<true>(img, fx, tcx & 0xFFFFu, sq[0], acx & 0xFFFFu);
+    d.y = decide_fast<true>(img, fx, tcx >> 16, sq[1], acx >> 16);
+    d.z = decide_fast<true>(img, fx, tcy & 0xFFFFu, sq[2], acy & 0xFFFFu);
+    d.w = decide_fast<true>(img, fx, tcy >> 16, sq[3], acy >> 16);
     const uint32_t rel = tile * WARP_TILE + lane * 4u;
     // PENDING slots are overwritten by the lane that resolves them, after a warp barrier
     __stcs(reinterpret_cast<uint4 *>(out + rel), d);
@@ -382,7 +386,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
         sq[0] = q.slo[i];
         slo_or |= sq[0];
         ta[0] = tk | (ac << 16);
-        d = decide_fast(img, fx, tk, sq[0], ac);
+        d = decide_fast<false>(img, fx, tk, sq[0], ac);
         out[rel] = d;
       }
       __syncwarp();
@@ -399,7 +403,7 @@ __global__ void __launch_bounds__(SELECT_THREADS, 1)
 select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint64_t per_cta) {
   extern __shared__ __align__(128) unsigned char smem[];   // [park lists][staged image]
   __shared__ __align__(8) unsigned long long mbar;
-  uint32_t *park = reinterpret_cast<uint32_t *>(smem);
+  uint4 *park = reinterpret_cast<uint4 *>(smem);
   unsigned char *staged = smem + PARK_BYTES;
   const uint64_t q0 = (uint64_t)blockIdx.x * per_cta;
   if (q0 >= n) return;

@@ -256,9 +256,9 @@ __device__ __forceinline__ void warp_prefix_count(const uint16_t *in, unsigned c
 __device__ __forceinline__ void write_dummy_task(const DeviceCatalog &c, uint32_t t) {
   const uint32_t T = c.n_tasks;
   if (threadIdx.x == 0) reinterpret_cast<uint32_t *>(c.image)[t] = dummy_header(T, c.nbw);
-  uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T)) + t * SLO_BUCKETS;
+  uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T) + t * REC_STRIDE);
   for (uint32_t j = threadIdx.x; j < SLO_BUCKETS; j += blockDim.x) rec[j] = 0u;
-  uint32_t *bm = reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(T)) + t * c.nbw;
+  uint32_t *bm = reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(T) + t * bitmap_stride(c.nbw));
   for (uint32_t j = threadIdx.x; j < c.nbw; j += blockDim.x) bm[j] = 0u;
 }
 
@@ -432,7 +432,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   };
 
   // SLO records (see common.cuh)
-  uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks)) + t * SLO_BUCKETS;
+  uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(c.n_tasks) + t * REC_STRIDE);
   // one bucket per thread of warps 16-23; lb = latencies in lower buckets: the lower warps'
   // buckets summed by the lanes, then a scan inside the warp
   if (first && tid >= B / 2 && tid < B / 2 + SLO_BUCKETS) {
@@ -462,7 +462,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
 
   // accuracy bitmap with running popcounts: warps 24-27, 128 words a round, same scheme; a
   // first segment's bitmap goes into the fixed part of the image
-  uint32_t *bitmap = first ? reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(c.n_tasks)) + t * nbw
+  uint32_t *bitmap = first ? reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(c.n_tasks) + t * bitmap_stride(nbw))
                            : reinterpret_cast<uint32_t *>(blk + BL.bitmap);
   if (tid >= 3 * B / 4 && tid < 3 * B / 4 + 128u) {
     const uint32_t lane = tid & 31u;
@@ -521,7 +521,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   });
 
   if (tid == 0) {
-    if (first) reinterpret_cast<uint32_t *>(c.image)[t] = ((base + BL.t2) >> 2) | (width << 24);
+    if (first) reinterpret_cast<uint32_t *>(c.image)[t] = (base + BL.t2) | (width << 24);
     else c.xhdr[xi] = make_uint4(base + BL.t2, width, base + BL.bitmap, 0u);
     c.slow[first ? t : c.n_tasks + xi] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs | (next << 8));
   }
