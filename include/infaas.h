@@ -293,6 +293,17 @@ int infaas_tally_static(const uint32_t *d_decision, uint64_t n, uint32_t n_varia
                         uint32_t *d_count, uint64_t *d_counters, int cuda_device,
                         void *cuda_stream);
 
+/* Measurement aid, not a step of the path: runs a kernel of independent 32-bit integer
+ * add / xor / compare / conditional-add chains on every multiprocessor of `cuda_device`
+ * (`iters` steps per chain, 1 .. 2^24) and reports in *h_lane_ops (HOST) how many
+ * lane-operations the launch executes.  Timed by the caller with CUDA events on
+ * `cuda_stream`, it gives the integer-pipe rate against which the feasibility scan of
+ * Section 4.1's per-query search (2 compares and 1 AND per variant examined) is put.
+ * d_sink: DEVICE, one u32, never written in practice.  Asynchronous, allocates nothing.
+ * Errors: E_NULL, E_BAD_ARG, E_CUDA. */
+int infaas_intpipe_probe(uint32_t iters, uint32_t *d_sink, int cuda_device, uint64_t *h_lane_ops,
+                         void *cuda_stream);
+
 /* Release the catalog and its device memory.  NULL is allowed. */
 void infaas_catalog_free(infaas_catalog *c);
 

@@ -40,6 +40,7 @@
 // Arithmetic: unsigned integers only.  Latency in microseconds (u32), accuracy in basis
 // points (u16), cost in integer units (u32).
 
+#include <algorithm>
 #include <cstdint>
 #include <cstring>
 #include <thread>
@@ -415,6 +416,81 @@ void oracle_assign_workers(const void *rows_v, uint32_t n_variants, const uint32
     }
     if (have) worker[q] = (uint32_t)best_w;
   }
+}
+
+// ---- scan-operation count (a measurement aid for the benchmark, not part of the method) ----
+// The cheapest feasible variant can be found by scanning, in (cost, pred, 10000-acc, id) order,
+// only the variants of the task that no other variant of it dominates -- B is dominated by A when
+// pred(A) <= pred(B), acc(A) >= acc(B), cost(A) <= cost(B) and one of the three is strict or
+// id(A) < id(B): whenever B is feasible so is A, and A sorts first.  oracle_frontier writes that
+// list for one task.  oracle_scan_ops charges every query the integer operations such a scan
+// needs, 32 entries at a time:
+//   feasible decision found at 1-based position pos:  3 * 32 * ceil(pos / 32)   (2 compares and
+//       1 AND per entry looked at)
+//   nothing feasible:  3 * F + 6 * F   (the whole list once for feasibility, once for the 64-bit
+//       distance, counted as 6 operations per entry)
+//   invalid query: 0
+// pos_out (may be NULL) receives each query's 0-based list position, 0xFFFFFFFF where there is none.
+static std::vector<uint32_t> frontier_of(const Row *rows, const uint32_t *queued,
+                                         const std::vector<uint32_t> &members) {
+  std::vector<uint32_t> keep;
+  for (uint32_t b : members) {
+    const uint32_t pb = pred_lat(rows[b].lat_us, queued[b], rows[b].batch);
+    bool dominated = false;
+    for (uint32_t a : members) {
+      if (a == b) continue;
+      const uint32_t pa = pred_lat(rows[a].lat_us, queued[a], rows[a].batch);
+      if (pa <= pb && rows[a].acc_bp >= rows[b].acc_bp && rows[a].cost <= rows[b].cost &&
+          (pa < pb || rows[a].acc_bp > rows[b].acc_bp || rows[a].cost < rows[b].cost || a < b)) {
+        dominated = true;
+        break;
+      }
+    }
+    if (!dominated) keep.push_back(b);
+  }
+  std::sort(keep.begin(), keep.end(), [&](uint32_t x, uint32_t y) {
+    Key kx{{0, rows[x].cost, pred_lat(rows[x].lat_us, queued[x], rows[x].batch), (uint64_t)(10000 - (int)rows[x].acc_bp), x}};
+    Key ky{{0, rows[y].cost, pred_lat(rows[y].lat_us, queued[y], rows[y].batch), (uint64_t)(10000 - (int)rows[y].acc_bp), y}};
+    return key_less(kx, ky);
+  });
+  return keep;
+}
+
+uint32_t oracle_frontier(const void *rows_v, uint32_t n_variants, uint32_t n_tasks, const uint32_t *queued,
+                         uint32_t task, uint32_t *ids_out, uint32_t cap) {
+  const Row *rows = (const Row *)rows_v;
+  auto members = members_by_task(rows, n_variants, n_tasks);
+  if (task >= n_tasks) return 0;
+  auto f = frontier_of(rows, queued, members[task]);
+  for (uint32_t i = 0; i < f.size() && i < cap; ++i) ids_out[i] = f[i];
+  return (uint32_t)f.size();
+}
+
+uint64_t oracle_scan_ops(const void *rows_v, uint32_t n_variants, uint32_t n_tasks, const uint32_t *queued,
+                         const uint16_t *task, const uint32_t *decision, uint64_t n, uint32_t *pos_out) {
+  const Row *rows = (const Row *)rows_v;
+  auto members = members_by_task(rows, n_variants, n_tasks);
+  std::vector<std::vector<uint32_t>> lists(n_tasks);
+  std::vector<uint32_t> pos_of(n_variants, 0xFFFFFFFFu);
+  for (uint32_t t = 0; t < n_tasks; ++t) {
+    lists[t] = frontier_of(rows, queued, members[t]);
+    for (uint32_t i = 0; i < lists[t].size(); ++i) pos_of[lists[t][i]] = i;
+  }
+  uint64_t ops = 0;
+  for (uint64_t q = 0; q < n; ++q) {
+    const uint32_t d = decision[q];
+    uint32_t pos = 0xFFFFFFFFu;
+    if (d != INVALID && task[q] < n_tasks) {
+      const uint64_t F = lists[task[q]].size();
+      if (d & NO_FEASIBLE_BIT) ops += 9 * F;
+      else if (d < n_variants && pos_of[d] != 0xFFFFFFFFu) {
+        pos = pos_of[d];
+        ops += 3ull * 32ull * ((uint64_t)pos / 32 + 1);
+      }
+    }
+    if (pos_out) pos_out[q] = pos;
+  }
+  return ops;
 }
 
 }  // extern "C"

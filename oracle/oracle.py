@@ -70,6 +70,12 @@ def _load():
         lib.oracle_assign_workers.argtypes = [ctypes.c_void_p, ctypes.c_uint32] + [ctypes.c_void_p] * 3 + \
             [ctypes.c_uint32] + [ctypes.c_void_p] * 2 + [ctypes.c_uint32, ctypes.c_void_p, ctypes.c_uint64,
                                                          ctypes.c_void_p]
+        lib.oracle_frontier.restype = ctypes.c_uint32
+        lib.oracle_frontier.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_void_p,
+                                        ctypes.c_uint32, ctypes.c_void_p, ctypes.c_uint32]
+        lib.oracle_scan_ops.restype = ctypes.c_uint64
+        lib.oracle_scan_ops.argtypes = [ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_void_p,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint64, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -117,6 +123,24 @@ class OracleCatalog:
         _load().oracle_load_update(_ptr(self.rows), self.n_variants, _ptr(self.queued),
                                    _ptr(self.served_total), _ptr(self.counters),
                                    _ptr(decision), decision.shape[0], int(window_us))
+
+    def frontier(self, task: int) -> np.ndarray:
+        """Ids of the task's non-dominated variants in (cost, pred, -acc, id) order at the current load."""
+        ids = np.empty(max(1, self.n_variants), np.uint32)
+        ln = _load().oracle_frontier(_ptr(self.rows), self.n_variants, self.n_tasks, _ptr(self.queued),
+                                     int(task), _ptr(ids), ids.shape[0])
+        return ids[:ln].copy()
+
+    def scan_ops(self, task, decision, want_pos: bool = False):
+        """Integer operations a 32-wide scan of the pruned lists needs for these decisions (see
+        oracle_scan_ops in infaas_oracle.cpp); with want_pos also every query's list position."""
+        task = np.ascontiguousarray(task, np.uint16)
+        decision = np.ascontiguousarray(decision, np.uint32)
+        pos = np.empty(task.shape[0], np.uint32) if want_pos else None
+        ops = _load().oracle_scan_ops(_ptr(self.rows), self.n_variants, self.n_tasks, _ptr(self.queued),
+                                      _ptr(task), _ptr(decision), task.shape[0],
+                                      _ptr(pos) if want_pos else None)
+        return (int(ops), pos) if want_pos else int(ops)
 
 
 class StatefulOracleCatalog(OracleCatalog):

@@ -24,6 +24,7 @@ _lib = None
 EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
            "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info",
+           "infaas_intpipe_probe",
            "infaas_tally", "infaas_pending_counts", "infaas_advance",
            "infaas_catalog_set_states", "infaas_catalog_get_states",
            "infaas_autoscale_config", "infaas_autoscale_step",
@@ -76,6 +77,8 @@ def _load():
     lib.infaas_workers_config.restype = lib.infaas_assign_workers.restype = i32
     lib.infaas_tally_static.argtypes = [vp, u64, u32, vp, vp, i32, vp]
     lib.infaas_tally_static.restype = i32
+    lib.infaas_intpipe_probe.argtypes = [u32, vp, i32, ctypes.POINTER(u64), vp]
+    lib.infaas_intpipe_probe.restype = i32
     lib.infaas_strerror.argtypes = [i32]
     lib.infaas_strerror.restype = ctypes.c_char_p
     lib.infaas_last_cuda_error.argtypes = []
@@ -256,6 +259,15 @@ def infaas_catalog_get_frontier(cat: Catalog, task: int, stream=None) -> np.ndar
                                                ctypes.byref(ln), _stream_ptr(stream)),
            "infaas_catalog_get_frontier")
     return ids[:ln.value].copy()
+
+
+def infaas_intpipe_probe(iters: int, d_sink, stream=None) -> int:
+    """Launches the integer-pipe probe on d_sink's device (see include/infaas.h); returns the
+    number of lane-operations the launch executes.  The caller times it with CUDA events."""
+    ops = ctypes.c_uint64(0)
+    _check(_load().infaas_intpipe_probe(int(iters), _dev_ptr(d_sink, "u32"), d_sink.device.index,
+                                        ctypes.byref(ops), _stream_ptr(stream)), "infaas_intpipe_probe")
+    return int(ops.value)
 
 
 def infaas_tally_static(d_decision, n_variants: int, d_count, d_counters, n=None, stream=None) -> None:

@@ -39,6 +39,18 @@ int cuda_fail(cudaError_t e) {
   return INFAAS_E_CUDA;
 }
 
+// Multiprocessors of a device, asked once per device.
+int sm_count_of(int device) {
+  static int cached[64] = {};
+  if (device < 0 || device >= 64) return 0;
+  if (!cached[device]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return 0;
+    cached[device] = n;
+  }
+  return cached[device];
+}
+
 #define CUDA_TRY(expr)                         \
   do {                                         \
     cudaError_t e__ = (expr);                  \
@@ -89,7 +101,23 @@ int refresh_select_plan(infaas_catalog *c, cudaStream_t stream) {
 
 }  // namespace
 
+int infaas::record_cuda_error(cudaError_t e) { return cuda_fail(e); }
+
 extern "C" {
+
+int infaas_intpipe_probe(uint32_t iters, uint32_t *d_sink, int cuda_device, uint64_t *h_lane_ops,
+                         void *cuda_stream) {
+  if (!d_sink || !h_lane_ops) return INFAAS_E_NULL;
+  if (iters == 0 || iters > (1u << 24)) return INFAAS_E_BAD_ARG;
+  DeviceScope scope(cuda_device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  const int sms = sm_count_of(cuda_device);
+  if (sms <= 0) return cuda_fail(cudaErrorInvalidDevice);
+  unsigned long long ops = 0;
+  CUDA_TRY(infaas::launch_intpipe_probe(iters, 0x9E3779B1u, d_sink, sms, &ops, static_cast<cudaStream_t>(cuda_stream)));
+  *h_lane_ops = ops;
+  return INFAAS_OK;
+}
 
 const char *infaas_strerror(int code) {
   switch (code) {
@@ -312,7 +340,7 @@ int infaas_tally(infaas_catalog *c, const uint32_t *d_decision, uint64_t n, void
   if (n > 0 && !aligned16(d_decision)) return INFAAS_E_ALIGN;
   DeviceScope scope(c->device);
   if (scope.status != cudaSuccess) return cuda_fail(scope.status);
-  CUDA_TRY(infaas::launch_tally(c->d, d_decision, n, static_cast<cudaStream_t>(cuda_stream)));
+  CUDA_TRY(infaas::launch_tally(c->d, d_decision, n, c->sm_count, static_cast<cudaStream_t>(cuda_stream)));
   return INFAAS_OK;
 }
 

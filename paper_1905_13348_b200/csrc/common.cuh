@@ -219,7 +219,7 @@ cudaError_t prepare_rebuild_kernel();
 cudaError_t launch_rebuild(const DeviceCatalog &c, bool advance_queues, uint32_t window_us,
                            cudaStream_t stream);
 cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uint64_t n,
-                         cudaStream_t stream);
+                         int sm_count, cudaStream_t stream);
 // Shared memory the launcher actually reserves for the image when asked for `image_smem`.
 uint32_t select_image_smem(uint32_t image_smem);
 // `image_smem`: bytes of dynamic shared memory reserved for the staged image (multiple of
@@ -250,5 +250,14 @@ cudaError_t launch_workers_build(uint32_t n_variants, const unsigned char *hw_by
 cudaError_t launch_assign_workers(const uint32_t *d_decision, uint64_t n, uint32_t n_variants,
                                   const uint32_t *worker_of, uint32_t *d_worker, int sm_count,
                                   cudaStream_t stream);
+
+// Integer-pipe probe: two CTAs per SM run `iters` steps of independent add / xor / compare /
+// conditional-add chains; *lane_ops receives the number of lane-operations the launch executes.
+cudaError_t launch_intpipe_probe(uint32_t iters, uint32_t seed, uint32_t *d_sink, int sm_count,
+                                 unsigned long long *lane_ops, cudaStream_t stream);
+
+// Remembers a CUDA error's text for infaas_last_cuda_error() (calling thread) and clears the
+// runtime's error state; returns INFAAS_E_CUDA.
+int record_cuda_error(cudaError_t e);
 
 }  // namespace infaas

@@ -16,6 +16,7 @@ static __device__ __align__(256) StaticScratch g_tally_scratch;
 constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 StaticScratch *g_scratch_addr[kMaxDevices] = {};   // device address of the array, per device
+int g_sm_count[kMaxDevices] = {};                  // multiprocessors, per device
 
 }  // namespace
 
@@ -29,8 +30,9 @@ extern "C" int infaas_tally_static(const uint32_t *d_decision, uint64_t n, uint3
   if (cuda_device < 0 || cuda_device >= kMaxDevices) return INFAAS_E_TOO_LARGE;
 
   int prev = -1;
-  if (cudaGetDevice(&prev) != cudaSuccess) return INFAAS_E_CUDA;
-  if (prev != cuda_device && cudaSetDevice(cuda_device) != cudaSuccess) return INFAAS_E_CUDA;
+  cudaError_t e = cudaGetDevice(&prev);
+  if (e != cudaSuccess) return infaas::record_cuda_error(e);
+  if (prev != cuda_device && (e = cudaSetDevice(cuda_device)) != cudaSuccess) return infaas::record_cuda_error(e);
   int rc = INFAAS_OK;
   StaticScratch *scratch = nullptr;
   {
@@ -39,10 +41,18 @@ extern "C" int infaas_tally_static(const uint32_t *d_decision, uint64_t n, uint3
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_scratch_addr[cuda_device]) {
       void *p = nullptr;
+      int sms = 0;
       // (the tally kernels' shared-memory limit is a per-device attribute, set here too)
-      if (cudaGetSymbolAddress(&p, g_tally_scratch) != cudaSuccess || !p ||
-          infaas::prepare_rebuild_kernel() != cudaSuccess) rc = INFAAS_E_CUDA;
-      else g_scratch_addr[cuda_device] = static_cast<StaticScratch *>(p);
+      if ((e = cudaGetSymbolAddress(&p, g_tally_scratch)) != cudaSuccess ||
+          (e = infaas::prepare_rebuild_kernel()) != cudaSuccess ||
+          (e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cuda_device)) != cudaSuccess) {
+        rc = infaas::record_cuda_error(e);
+      } else if (!p || sms <= 0) {
+        rc = infaas::record_cuda_error(cudaErrorInvalidSymbol);
+      } else {
+        g_scratch_addr[cuda_device] = static_cast<StaticScratch *>(p);
+        g_sm_count[cuda_device] = sms;
+      }
     }
     scratch = g_scratch_addr[cuda_device];
   }
@@ -53,14 +63,13 @@ extern "C" int infaas_tally_static(const uint32_t *d_decision, uint64_t n, uint3
     view.n_variants = n_variants;
     view.count_by_id = scratch->count;
     view.counters = scratch->counters;
-    if (cudaMemsetAsync(scratch, 0, (size_t)n_variants * 4, s) != cudaSuccess ||
-        cudaMemsetAsync(scratch->counters, 0, sizeof(scratch->counters), s) != cudaSuccess ||
-        infaas::launch_tally(view, d_decision, n, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_count, scratch->count, (size_t)n_variants * 4, cudaMemcpyDeviceToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(d_counters, scratch->counters, 24, cudaMemcpyDeviceToDevice, s) != cudaSuccess)
-      rc = INFAAS_E_CUDA;
+    if ((e = cudaMemsetAsync(scratch, 0, (size_t)n_variants * 4, s)) != cudaSuccess ||
+        (e = cudaMemsetAsync(scratch->counters, 0, sizeof(scratch->counters), s)) != cudaSuccess ||
+        (e = infaas::launch_tally(view, d_decision, n, g_sm_count[cuda_device], s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d_count, scratch->count, (size_t)n_variants * 4, cudaMemcpyDeviceToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(d_counters, scratch->counters, 24, cudaMemcpyDeviceToDevice, s)) != cudaSuccess)
+      rc = infaas::record_cuda_error(e);   // the text is kept for infaas_last_cuda_error()
   }
-  if (rc == INFAAS_E_CUDA) (void)cudaGetLastError();
   if (prev != cuda_device) (void)cudaSetDevice(prev);
   return rc;
 }

@@ -849,7 +849,7 @@ constexpr uint32_t TALLY_SMEM_MAX_PARTS = 8;           // beyond this many id ra
 constexpr uint64_t TALLY_SMEM_MIN_N = 1u << 18;        // below this the zero/flush passes cost more than they save
 
 cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uint64_t n,
-                         cudaStream_t stream) {
+                         int sm_count, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
   const uint32_t parts = (c.n_variants + TALLY_SMEM_MAX_VARIANTS - 1) / TALLY_SMEM_MAX_VARIANTS;
   if (n >= TALLY_SMEM_MIN_N && parts <= TALLY_SMEM_MAX_PARTS) {
@@ -857,7 +857,7 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
     const size_t smem = (size_t)(bins + 32) * 4;                 // 32 spare bins
     const uint32_t per_sm = smem > 100 * 1024 ? 1 : 2;
     uint64_t want = ((n >> 2) + TALLY_SMEM_THREADS * 8 - 1) / (TALLY_SMEM_THREADS * 8);
-    uint64_t shares = (uint64_t)148 * per_sm / parts;          // CTAs per id range
+    uint64_t shares = (uint64_t)sm_count * per_sm / parts;     // CTAs per id range
     if (shares > want) shares = want;
     if (shares < 1) shares = 1;
     tally_smem_kernel<<<(uint32_t)(shares * parts), TALLY_SMEM_THREADS, smem, stream>>>(
@@ -865,7 +865,8 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
     return cudaGetLastError();
   }
   uint64_t want = ((n >> 2) + 255) / 256;
-  uint32_t grid = (uint32_t)(want < 1 ? 1 : (want > 148 * 8 ? 148 * 8 : want));
+  const uint64_t most = (uint64_t)sm_count * 8;
+  uint32_t grid = (uint32_t)(want < 1 ? 1 : (want > most ? most : want));
   tally_kernel<<<grid, 256, 0, stream>>>(d_decision, n, c.n_variants, c.count_by_id, c.counters);
   return cudaGetLastError();
 }

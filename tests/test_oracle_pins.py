@@ -266,3 +266,48 @@ def test_saturating_queue_and_extreme_queries():
     d = o.select(np.array([0, 0, 0, 1], np.uint16), np.array([0, 2**32 - 1, 1, 5], np.uint32),
                  np.array([0, 10001, 10000, 0], np.uint16))
     assert list(d) == [NO_FEASIBLE_BIT | 1, NO_FEASIBLE_BIT | 1, 1, INVALID]
+
+
+# -- the pruned list behind the benchmark's scan-operation count: checked against the dominance
+#    definition in plain Python, and against the brute-force oracle (first feasible entry of the
+#    list = the oracle's decision, which never prunes) ---------------------------------------
+@pytest.mark.parametrize("seed", range(4))
+def test_frontier_and_scan_ops(seed):
+    rng = np.random.default_rng(900 + seed)
+    nv, n_tasks = int(rng.integers(20, 60)), 2
+    rows = rows_from(rng.integers(0, n_tasks, nv), rng.choice([1, 2, 4], nv), rng.integers(1, 30, nv),
+                     rng.integers(6995, 7005, nv), rng.integers(1, 6, nv), rng.integers(0, 4, nv))
+    o = OracleCatalog(rows, n_tasks)
+    pred = [py_pred(int(r["lat_us"]), int(r["queued"]), int(r["batch"])) for r in rows]
+    attr = [(pred[v], -int(rows["acc_bp"][v]), int(rows["cost"][v])) for v in range(nv)]
+
+    def dominates(a, b):
+        return a != b and all(x <= y for x, y in zip(attr[a], attr[b])) and (attr[a] != attr[b] or a < b)
+
+    lists = []
+    for t in range(n_tasks):
+        mem = [v for v in range(nv) if int(rows["task"][v]) == t]
+        want = sorted([b for b in mem if not any(dominates(a, b) for a in mem)],
+                      key=lambda v: (attr[v][2], attr[v][0], attr[v][1], v))
+        got = [int(x) for x in o.frontier(t)]
+        assert got == want
+        lists.append(got)
+    n = 3000
+    task = rng.integers(0, n_tasks + 1, n).astype(np.uint16)
+    slo, acc = rng.integers(0, 70, n).astype(np.uint32), rng.integers(6990, 7010, n).astype(np.uint16)
+    d = o.select(task, slo, acc)
+    ops, pos = o.scan_ops(task, d, want_pos=True)
+    total = 0
+    for q in range(n):
+        if task[q] >= n_tasks or d[q] == INVALID:
+            assert pos[q] == 0xFFFFFFFF
+            continue
+        L = lists[int(task[q])]
+        first = next((i for i, v in enumerate(L) if pred[v] <= slo[q] and rows["acc_bp"][v] >= acc[q]), None)
+        if d[q] >> 31:
+            assert first is None and pos[q] == 0xFFFFFFFF
+            total += 9 * len(L)
+        else:
+            assert first is not None and L[first] == int(d[q]) and pos[q] == first
+            total += 96 * (first // 32 + 1)
+    assert ops == total
