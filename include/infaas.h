@@ -137,6 +137,15 @@ int infaas_load_update(infaas_catalog *c, const uint32_t *d_decision, uint64_t n
  *                written (set = 0) or read (set = 1).
  * Asynchronous, stream-ordered, allocate nothing.  Errors: E_NULL, E_ALIGN, E_TOO_LARGE, E_CUDA. */
 int infaas_tally(infaas_catalog *c, const uint32_t *d_decision, uint64_t n, void *cuda_stream);
+
+/* infaas_select_batch followed by infaas_load_update over the same n queries, as one call
+ * (the arrival of a window of queries and the refresh of the load that follows it:
+ * Section 4.1 "Case I", then Section 4.2.2 / Section 5).  Same arguments, layouts, results and
+ * errors as the two calls; n <= 2^32-1.  For windows below 2^18 queries the selection kernel
+ * counts its own decisions, which saves the pass over d_decision and one kernel launch. */
+int infaas_select_update(infaas_catalog *c, const uint16_t *d_task, const uint32_t *d_slo_us,
+                         const uint16_t *d_min_acc_bp, uint64_t n, uint32_t *d_decision,
+                         uint32_t window_us, void *cuda_stream);
 int infaas_pending_counts(infaas_catalog *c, uint32_t *d_counts, int set, void *cuda_stream);
 int infaas_advance(infaas_catalog *c, uint32_t window_us, void *cuda_stream);
 

@@ -24,7 +24,7 @@ _lib = None
 EXPORTS = ("infaas_catalog_load", "infaas_select_batch", "infaas_load_update",
            "infaas_catalog_get_state", "infaas_catalog_get_frontier", "infaas_catalog_free",
            "infaas_strerror", "infaas_last_cuda_error", "infaas_tally_static", "infaas_catalog_get_info",
-           "infaas_intpipe_probe",
+           "infaas_intpipe_probe", "infaas_select_update",
            "infaas_tally", "infaas_pending_counts", "infaas_advance",
            "infaas_catalog_set_states", "infaas_catalog_get_states",
            "infaas_autoscale_config", "infaas_autoscale_step",
@@ -52,6 +52,8 @@ def _load():
     lib.infaas_catalog_load.argtypes = [vp, u32, u32, i32, ctypes.POINTER(vp)]
     lib.infaas_select_batch.argtypes = [vp, vp, vp, vp, u64, vp, vp]
     lib.infaas_load_update.argtypes = [vp, vp, u64, u32, vp]
+    lib.infaas_select_update.argtypes = [vp, vp, vp, vp, u64, vp, u32, vp]
+    lib.infaas_select_update.restype = i32
     lib.infaas_catalog_get_state.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.infaas_catalog_get_frontier.argtypes = [vp, u32, vp, u32, ctypes.POINTER(u32), vp]
     lib.infaas_catalog_get_info.argtypes = [vp, vp, vp]
@@ -152,6 +154,15 @@ def infaas_load_update(cat: Catalog, d_decision, window_us: int, n=None, stream=
     n = int(d_decision.shape[0]) if n is None else int(n)
     _check(_load().infaas_load_update(cat.handle, _dev_ptr(d_decision, "u32"), n, int(window_us),
                                       _stream_ptr(stream)), "infaas_load_update")
+
+
+def infaas_select_update(cat: Catalog, d_task, d_slo_us, d_min_acc_bp, d_decision, window_us: int, n=None,
+                         stream=None) -> None:
+    """One window: decide its queries, then fold the decisions into the load (one call)."""
+    n = int(d_task.shape[0]) if n is None else int(n)
+    _check(_load().infaas_select_update(cat.handle, _dev_ptr(d_task, "u16"), _dev_ptr(d_slo_us, "u32"),
+                                        _dev_ptr(d_min_acc_bp, "u16"), n, _dev_ptr(d_decision, "u32"),
+                                        int(window_us), _stream_ptr(stream)), "infaas_select_update")
 
 
 def infaas_tally(cat: Catalog, d_decision, n=None, stream=None) -> None:

@@ -329,7 +329,29 @@ int infaas_select_batch(infaas_catalog *c, const uint16_t *d_task, const uint32_
   DeviceScope scope(c->device);
   if (scope.status != cudaSuccess) return cuda_fail(scope.status);
   CUDA_TRY(infaas::launch_select(c->d, d_task, d_slo_us, d_min_acc_bp, n, d_decision, c->sm_count,
-                                 c->select_smem, static_cast<cudaStream_t>(cuda_stream)));
+                                 c->select_smem, /*tally=*/false, static_cast<cudaStream_t>(cuda_stream)));
+  return INFAAS_OK;
+}
+
+int infaas_select_update(infaas_catalog *c, const uint16_t *d_task, const uint32_t *d_slo_us,
+                         const uint16_t *d_min_acc_bp, uint64_t n, uint32_t *d_decision,
+                         uint32_t window_us, void *cuda_stream) {
+  if (!c) return INFAAS_E_NULL;
+  if (n > 0xFFFFFFFFull) return INFAAS_E_TOO_LARGE;
+  if (n == 0 || n >= infaas::FUSED_TALLY_MAX_N) {
+    // large batches: a pass of its own over the decisions with shared-memory histograms is cheaper
+    const int rc = infaas_select_batch(c, d_task, d_slo_us, d_min_acc_bp, n, d_decision, cuda_stream);
+    return rc != INFAAS_OK ? rc : infaas_load_update(c, d_decision, n, window_us, cuda_stream);
+  }
+  if (!d_task || !d_slo_us || !d_min_acc_bp || !d_decision) return INFAAS_E_NULL;
+  if (!aligned16(d_task) || !aligned16(d_slo_us) || !aligned16(d_min_acc_bp) || !aligned16(d_decision))
+    return INFAAS_E_ALIGN;
+  DeviceScope scope(c->device);
+  if (scope.status != cudaSuccess) return cuda_fail(scope.status);
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  CUDA_TRY(infaas::launch_select(c->d, d_task, d_slo_us, d_min_acc_bp, n, d_decision, c->sm_count,
+                                 c->select_smem, /*tally=*/true, s));
+  CUDA_TRY(infaas::launch_rebuild(c->d, /*advance_queues=*/true, window_us, s));
   return INFAAS_OK;
 }
 

@@ -224,10 +224,14 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
 uint32_t select_image_smem(uint32_t image_smem);
 // `image_smem`: bytes of dynamic shared memory reserved for the staged image (multiple of
 // 16).  If the image is larger at run time the kernel reads it from global memory instead.
+// `tally`: the kernel also adds the decisions to the pending per-variant counts and the
+// catalog's counters (what launch_tally would do with them).
 // Returns cudaErrorInvalidValue if n is too large for the launch geometry.
 cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const uint32_t *d_slo,
                           const uint16_t *d_min_acc, uint64_t n, uint32_t *d_decision,
-                          int sm_count, uint32_t image_smem, cudaStream_t stream);
+                          int sm_count, uint32_t image_smem, bool tally, cudaStream_t stream);
+// Batches below this size are tallied by the selection kernel itself in infaas_select_update.
+constexpr uint64_t FUSED_TALLY_MAX_N = 1u << 18;
 
 // Scaling-up step of the Model-Autoscaler for every task, from the pending per-variant
 // counts; s_inst / s_arch / s_qps (floor(10^9 * batch / lat_us)) are per slot, task_slo per

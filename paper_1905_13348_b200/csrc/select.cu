@@ -285,24 +285,52 @@ struct Park {
   uint32_t cnt;
 };
 
-// Resolve the 32 parked queries [first, first + count), one per lane.
-template <class Img>
+// Per-thread sums of the decisions tallied by the fused form of the kernel (feasible, nothing
+// feasible, invalid), added to the catalog's counters at the end.
+struct Tallies {
+  uint32_t feas = 0, nofeas = 0, inval = 0;
+};
+
+// Tally one decision per lane into the per-variant counts (Section 4.2.2: the load a variant
+// serves is tracked from the queries it is given): lanes of the warp that hold the same variant
+// share one atomic.  `live`: this lane holds a final decision.  All lanes call this together.
+__device__ __forceinline__ void tally_decision(const DeviceCatalog &c, uint32_t d, bool live, Tallies &tl) {
+  const bool feas = live && d < c.n_variants;                 // n_variants < 2^31: bit 31 clear
+  const bool inval = live && !feas && (d == INFAAS_INVALID || !(d & INFAAS_NO_FEASIBLE));
+  tl.feas += feas;
+  tl.inval += inval;
+  tl.nofeas += live && !feas && !inval;
+  const unsigned fm = __ballot_sync(0xFFFFFFFFu, feas);
+  if (feas) {
+    const unsigned peers = __match_any_sync(fm, d);
+    if ((threadIdx.x & 31u) == (uint32_t)__ffs(peers) - 1u) atomicAdd(&c.count_by_id[d], (uint32_t)__popc(peers));
+  }
+}
+
+// Resolve the parked queries [first, first + count), count <= 32, one per lane.
+template <bool Tally, class Img>
 __device__ __forceinline__ void resolve_parked(const Img &img, const DeviceCatalog &c, const Fixed &fx, uint32_t *out,
-                                               const Park &pk, uint32_t first, uint32_t count) {
+                                               const Park &pk, uint32_t first, uint32_t count, Tallies &tl) {
   const uint32_t lane = threadIdx.x & 31;
+  uint32_t d = 0;
   if (lane < count) {
     const uint4 e = pk.e[first + lane];
-    out[e.x] = decide_slow(img, c, fx, e.z & 0xFFFFu, e.y, e.z >> 16);
+    d = decide_slow(img, c, fx, e.z & 0xFFFFu, e.y, e.z >> 16);
+    out[e.x] = d;
+  }
+  if (Tally) {
+    __syncwarp();
+    tally_decision(c, d, lane < count, tl);
   }
 }
 
 // Park the queries a lane holds whose bit is set in `pm` (bit i = i-th of its four
 // queries, data in ta[i] / s[i], offset rel + i); flush whenever 32 are waiting.  All
 // lanes of the warp call this together.
-template <class Img>
+template <bool Tally, class Img>
 __device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatalog &c, const Fixed &fx, uint32_t *out, Park &pk,
                                                uint32_t pm, uint32_t rel, const uint32_t (&ta)[4],
-                                               const uint32_t (&s)[4]) {
+                                               const uint32_t (&s)[4], Tallies &tl) {
   const uint32_t lane_lt = (1u << (threadIdx.x & 31)) - 1u;
   unsigned m;
   while ((m = __ballot_sync(0xFFFFFFFFu, pm != 0u)) != 0u) {
@@ -317,17 +345,20 @@ __device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatal
     __syncwarp();
     if (pk.cnt >= 32) {
       pk.cnt -= 32;
-      resolve_parked(img, c, fx, out, pk, pk.cnt, 32);
+      resolve_parked<Tally>(img, c, fx, out, pk, pk.cnt, 32, tl);
       __syncwarp();
     }
   }
 }
 
-template <class Img>
+// `Tally`: also count the decisions per variant (the first half of the load update), for
+// batches small enough that a second pass over them would cost more than the atomics here.
+template <bool Tally, class Img>
 __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
                                             uint64_t q0, uint32_t span, uint4 *park_all, uint2 t4, uint4 s4,
                                             uint2 a4) {
   const Fixed fx = make_fixed(c);
+  Tallies tl;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Park pk;
   pk.e = park_all + warp * PARK_CAP;
@@ -365,13 +396,19 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
     const uint32_t rel = tile * WARP_TILE + lane * 4u;
     // PENDING slots are overwritten by the lane that resolves them, after a warp barrier
     __stcs(reinterpret_cast<uint4 *>(out + rel), d);
+    if (Tally) {                         // what is PENDING is tallied when it is resolved
+      tally_decision(c, d.x, d.x != PENDING, tl);
+      tally_decision(c, d.y, d.y != PENDING, tl);
+      tally_decision(c, d.z, d.z != PENDING, tl);
+      tally_decision(c, d.w, d.w != PENDING, tl);
+    }
     // valid ids stay below 2^31, PENDING has bit 31 set
     if (__any_sync(0xFFFFFFFFu, (int)(d.x | d.y | d.z | d.w) < 0)) {
       const uint32_t pm = (d.x >> 31) | ((d.y >> 31) << 1) | ((d.z >> 31) << 2) | ((d.w >> 31) << 3);
       const uint32_t ta[4] = {tq[0] | (aq[0] << 16), tq[1] | (aq[1] << 16), tq[2] | (aq[2] << 16),
                               tq[3] | (aq[3] << 16)};
       __syncwarp();
-      park_and_flush(img, c, fx, out, pk, pm, rel, ta, sq);
+      park_and_flush<Tally>(img, c, fx, out, pk, pm, rel, ta, sq, tl);
     }
   }
   // ragged tail of the CTA's range (fewer than WARP_TILE queries): one warp, scalar accesses
@@ -390,15 +427,26 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
         out[rel] = d;
       }
       __syncwarp();
-      park_and_flush(img, c, fx, out, pk, d >> 31, rel, ta, sq);
+      if (Tally) tally_decision(c, d, rel < span && d != PENDING, tl);
+      park_and_flush<Tally>(img, c, fx, out, pk, d >> 31, rel, ta, sq, tl);
     }
   }
   __syncwarp();
-  resolve_parked(img, c, fx, out, pk, 0, pk.cnt);
+  resolve_parked<Tally>(img, c, fx, out, pk, 0, pk.cnt, tl);
   slo_or = __reduce_or_sync(0xFFFFFFFFu, slo_or);
   if (lane == 0 && (slo_or & ~*c.slo_seen)) atomicOr(c.slo_seen, slo_or);
+  if (Tally) {
+    const uint32_t f = __reduce_add_sync(0xFFFFFFFFu, tl.feas), nf = __reduce_add_sync(0xFFFFFFFFu, tl.nofeas),
+                   iv = __reduce_add_sync(0xFFFFFFFFu, tl.inval);
+    if (lane == 0) {
+      if (f) atomicAdd(&c.counters[0], (unsigned long long)f);
+      if (nf) atomicAdd(&c.counters[1], (unsigned long long)nf);
+      if (iv) atomicAdd(&c.counters[2], (unsigned long long)iv);
+    }
+  }
 }
 
+template <bool Tally>
 __global__ void __launch_bounds__(SELECT_THREADS, 1)
 select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint64_t per_cta) {
   extern __shared__ __align__(128) unsigned char smem[];   // [park lists][staged image]
@@ -427,18 +475,21 @@ select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint6
       return;
     }
     SharedImage img{smem_u32(staged)};
-    select_body(img, c, q, q0, span, park, t4, s4, a4);
+    select_body<Tally>(img, c, q, q0, span, park, t4, s4, a4);
   } else {
     // the image does not fit in shared memory: read it from global memory (L1/L2 resident)
     GlobalImage img{c.image};
-    select_body(img, c, q, q0, span, park, t4, s4, a4);
+    select_body<Tally>(img, c, q, q0, span, park, t4, s4, a4);
   }
 }
 
 }  // namespace
 
 cudaError_t prepare_select_kernel() {
-  return cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(select_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)SELECT_MAX_SMEM);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)SELECT_MAX_SMEM);
 }
 
@@ -449,7 +500,7 @@ uint32_t select_image_smem(uint32_t image_smem) {
 
 cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const uint32_t *d_slo,
                           const uint16_t *d_min_acc, uint64_t n, uint32_t *d_decision,
-                          int sm_count, uint32_t image_smem, cudaStream_t stream) {
+                          int sm_count, uint32_t image_smem, bool tally, cudaStream_t stream) {
   if (n == 0) return cudaSuccess;
   image_smem = select_image_smem(image_smem);
   // one CTA per SM; every CTA takes one contiguous range, a multiple of the warp tile
@@ -461,8 +512,10 @@ cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const 
   grid = (n + per_cta - 1) / per_cta;
   if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
   Queries q{d_task, d_slo, d_min_acc, d_decision};
-  select_kernel<<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n,
-                                                                                     per_cta);
+  if (tally)
+    select_kernel<true><<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n, per_cta);
+  else
+    select_kernel<false><<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n, per_cta);
   return cudaGetLastError();
 }
 

@@ -256,8 +256,8 @@ def test_full_size_single_launch_then_update(name):
         cat.free()
 
 
-@pytest.mark.parametrize("name,state_every", [("C3", 16), ("C5", 100)])
-def test_full_size_windowed(name, state_every):
+@pytest.mark.parametrize("name,state_every,fused", [("C3", 16, False), ("C3", 32, True), ("C5", 100, False)])
+def test_full_size_windowed(name, state_every, fused):
     """The configuration as a stream of windows (select one window, update, repeat): every
     decision of every window is compared; the load state every `state_every` windows and at
     the end."""
@@ -272,8 +272,11 @@ def test_full_size_windowed(name, state_every):
     try:
         for k in range(nwin):
             s = slice(k * w.window, (k + 1) * w.window)
-            P.infaas_select_batch(cat, d_task[s], d_slo[s], d_acc[s], d_dec[s])
-            P.infaas_load_update(cat, d_dec[s], w.window_us)
+            if fused:
+                P.infaas_select_update(cat, d_task[s], d_slo[s], d_acc[s], d_dec[s], w.window_us)
+            else:
+                P.infaas_select_batch(cat, d_task[s], d_slo[s], d_acc[s], d_dec[s])
+                P.infaas_load_update(cat, d_dec[s], w.window_us)
             want = o.select(w.task[s], w.slo_us[s], w.min_acc_bp[s], _threads())
             o.load_update(want, w.window_us)
             got = _to_host_u32(d_dec[s])
@@ -282,6 +285,46 @@ def test_full_size_windowed(name, state_every):
             if (k + 1) % state_every == 0 or k == nwin - 1:
                 _assert_state_fast(cat, o, w.rows)
         assert int(o.counters.sum()) == w.n_queries
+    finally:
+        cat.free()
+
+
+@pytest.mark.parametrize("name,kw,sizes", [
+    ("C3", {"n_queries": 40_000}, [4096, 1, 0, 777, 8192, 130, 2049, 10_000, 14_654]),
+    ("C5", {"n_windows": 3, "window": 8192}, [8192, 5, 8187, 8192]),
+    ("C4", {"n_queries": 30_000}, [30_000]),
+    ("C2", {"n_queries": 300_000}, [100, 299_900]),          # the second window is above the fused limit
+])
+def test_fused_window_call(name, kw, sizes):
+    """infaas_select_update (one call per window; the selection kernel tallies its own decisions
+    for small windows) against the oracle: decisions of every window, state after every window.
+    Ragged and empty windows, bad tasks in between, heavy load so that the lists move."""
+    import paper_1905_13348_b200 as P
+    torch = _torch()
+    w = W.make(name, **kw)
+    assert sum(sizes) <= w.n_queries
+    task = w.task.copy()
+    task[::97] = w.n_tasks + 3                                   # invalid queries are counted too
+    window_us = 500
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = OracleCatalog(w.rows, w.n_tasks)
+    try:
+        lo = 0
+        for n in sizes:
+            s = slice(lo, lo + n)
+            d_dec = torch.empty(n, dtype=torch.int32, device="cuda")     # fresh arrays: 16-byte aligned
+            if n:
+                P.infaas_select_update(cat, _to_dev(task[s]), _to_dev(w.slo_us[s]), _to_dev(w.min_acc_bp[s]),
+                                       d_dec, window_us)
+            else:
+                P.infaas_select_update(cat, None, None, None, None, window_us, n=0)
+            want = o.select(task[s], w.slo_us[s], w.min_acc_bp[s], _threads())
+            o.load_update(want, window_us)
+            got = _to_host_u32(d_dec)
+            bad = np.flatnonzero(got != want)
+            assert bad.size == 0, (name, lo, n, bad[:5], got[bad[:5]], want[bad[:5]])
+            assert_state_equal(cat, o)
+            lo += n
     finally:
         cat.free()
 
