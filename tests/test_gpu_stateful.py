@@ -65,6 +65,55 @@ def test_configs_reduced_stateful(name, kw, p, load_hi):
     assert seen[0] > 0 and seen[1] > 0 and seen[2] > 0, seen
 
 
+def test_full_size_stateful_two_launches():
+    """The 16M-query configuration with the benchmark leg's state mix: one launch over all 2^24
+    queries, the load update (states move), and a second launch -- every decision of both."""
+    import paper_1905_13348_b200 as P
+    from tests.test_gpu_parity import _to_dev
+    w = W.make("C3")
+    state, load = W.variant_states(w.n_variants)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    o = StatefulOracleCatalog(w.rows, w.n_tasks, state, load)
+    window_us = 256 * w.window_us
+    try:
+        P.infaas_catalog_set_states(cat, state, load)
+        d_task, d_slo, d_acc = _to_dev(w.task), _to_dev(w.slo_us), _to_dev(w.min_acc_bp)
+        for launch in range(2):
+            d_dec = gpu_select(cat, w.task, w.slo_us, w.min_acc_bp) if launch == 0 else d_dec
+            if launch:
+                P.infaas_select_batch(cat, d_task, d_slo, d_acc, d_dec)
+            want = o.select(w.task, w.slo_us, w.min_acc_bp, 16)
+            got = _to_host_u32(d_dec)
+            bad = np.flatnonzero(got != want)
+            assert bad.size == 0, (launch, bad[:5], got[bad[:5]], want[bad[:5]])
+            P.infaas_load_update(cat, d_dec, window_us)
+            o.load_update(want, window_us)
+            assert np.array_equal(P.infaas_catalog_get_state(cat)["queued"], o.queued)
+            assert np.array_equal(P.infaas_catalog_get_states(cat), o.state)
+        assert (o.state != state).any()                       # the update did move states
+    finally:
+        cat.free()
+
+
+def test_stateful_catalog_whose_image_exceeds_shared_memory():
+    """A state-aware catalog large enough that the selection kernel reads its tables from
+    global memory (128 tasks x 512 variants, both lists long): three windows, all decisions."""
+    import paper_1905_13348_b200 as P
+    w = W.make("C5", n_windows=3)
+    rng = np.random.default_rng(35)
+    state = _states(rng, w.n_variants, (0.45, 0.45, 0.05, 0.05))
+    load = rng.integers(0, 50_000, w.n_variants).astype(np.uint32)
+    cat = P.infaas_catalog_load(w.rows, w.n_tasks)
+    try:
+        P.infaas_catalog_set_states(cat, state, load)
+        info = P.infaas_catalog_get_info(cat)
+        assert info["image_bytes"] > info["image_smem"], info
+    finally:
+        cat.free()
+    seen = run_stateful(w, state, load, n_threads=16)
+    assert seen[0] > 0 and seen[1] > 0
+
+
 def test_states_follow_the_load_over_many_windows():
     # little drain per window: variants overload, queries move on to Inactive ones, which
     # become Active (and overload in turn), then everything drains

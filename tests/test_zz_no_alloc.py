@@ -45,6 +45,33 @@ def test_static_tally_matches_load_update_twice():
     cat.free()
 
 
+def test_static_tally_large_batch_near_the_size_limit():
+    """A batch large enough for the shared-memory histogram kernel over a catalog just below
+    the array's limit (the ids are counted in two ranges then), against numpy, twice."""
+    import torch
+
+    import paper_1905_13348_b200 as P
+
+    nv = 60_001
+    rng = np.random.default_rng(22)
+    d_count = torch.full((nv,), -1, dtype=torch.int32, device="cuda")
+    d_counters = torch.full((3,), -1, dtype=torch.int64, device="cuda")
+    for n in ((1 << 18) + 13, (1 << 19) + 1):
+        dec = rng.integers(0, nv, n).astype(np.uint32)
+        dec[::7] |= 0x80000000
+        dec[::31] = 0xFFFFFFFF
+        dec[5::41] = nv + 5
+        dec[1000:60000] = nv - 1                     # a hot variant in the upper range
+        d_dec = torch.from_numpy(dec.view(np.int32)).cuda()
+        P.infaas_tally_static(d_dec, nv, d_count, d_counters)
+        torch.cuda.synchronize()
+        feas = dec[dec < nv]
+        assert np.array_equal(d_count.cpu().numpy().view(np.uint32), np.bincount(feas, minlength=nv).astype(np.uint32))
+        flagged = ((dec >> 31) == 1) & (dec != 0xFFFFFFFF)
+        want = [feas.size, int(flagged.sum()), int(n - feas.size - flagged.sum())]
+        assert d_counters.cpu().numpy().tolist() == want
+
+
 def test_static_tally_rejects_sizes_beyond_its_array():
     import torch
 
