@@ -111,10 +111,11 @@ struct Fixed {
   uint32_t bm_stride;         // bytes of one bitmap
   uint32_t acc_lo, acc_hi;    // accuracy window, both ends included
 };
-__device__ __forceinline__ Fixed make_fixed(const DeviceCatalog &c) {
+// `hdr`: the words the last rebuild published (image bytes, bucket scale, -bmin).
+__device__ __forceinline__ Fixed make_fixed(const DeviceCatalog &c, const uint4 hdr) {
   Fixed f;
-  f.scale = __uint_as_float(c.image_hdr[1]);
-  f.neg_bmin = __uint_as_float(c.image_hdr[2]);
+  f.scale = __uint_as_float(hdr.y);
+  f.neg_bmin = __uint_as_float(hdr.z);
   f.n_tasks = c.n_tasks;
   f.rec_off = image_rec_offset(c.n_tasks);
   f.bm_off = image_bitmap_offset(c.n_tasks) - 4u * (c.acc_lo / ACC_WORD_BITS);
@@ -355,9 +356,9 @@ __device__ __forceinline__ void park_and_flush(const Img &img, const DeviceCatal
 // batches small enough that a second pass over them would cost more than the atomics here.
 template <bool Tally, class Img>
 __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog &c, const Queries &q,
-                                            uint64_t q0, uint32_t span, uint4 *park_all, uint2 t4, uint4 s4,
-                                            uint2 a4) {
-  const Fixed fx = make_fixed(c);
+                                            uint64_t q0, uint32_t span, uint4 *park_all, const uint4 hdr,
+                                            uint32_t slo_seen, uint2 t4, uint4 s4, uint2 a4) {
+  const Fixed fx = make_fixed(c, hdr);
   Tallies tl;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   Park pk;
@@ -434,7 +435,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
   __syncwarp();
   resolve_parked<Tally>(img, c, fx, out, pk, 0, pk.cnt, tl);
   slo_or = __reduce_or_sync(0xFFFFFFFFu, slo_or);
-  if (lane == 0 && (slo_or & ~*c.slo_seen)) atomicOr(c.slo_seen, slo_or);
+  if (lane == 0 && (slo_or & ~slo_seen)) atomicOr(c.slo_seen, slo_or);
   if (Tally) {
     const uint32_t f = __reduce_add_sync(0xFFFFFFFFu, tl.feas), nf = __reduce_add_sync(0xFFFFFFFFu, tl.nofeas),
                    iv = __reduce_add_sync(0xFFFFFFFFu, tl.inval);
@@ -448,7 +449,7 @@ __device__ __forceinline__ void select_body(const Img &img, const DeviceCatalog 
 
 template <bool Tally>
 __global__ void __launch_bounds__(SELECT_THREADS, 1)
-select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint64_t per_cta) {
+select_kernel(DeviceCatalog c, uint32_t stage_bytes, Queries q, uint64_t n, uint64_t per_cta) {
   extern __shared__ __align__(128) unsigned char smem[];   // [park lists][staged image]
   __shared__ __align__(8) unsigned long long mbar;
   uint4 *park = reinterpret_cast<uint4 *>(smem);
@@ -456,10 +457,13 @@ select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint6
   const uint64_t q0 = (uint64_t)blockIdx.x * per_cta;
   if (q0 >= n) return;
   const uint32_t span = (uint32_t)min(n - q0, per_cta);     // <= MAX_SPAN (checked by the launcher)
-  const uint32_t bytes = c.image_hdr[0];
-  const bool in_smem = bytes <= image_smem;
-  if (in_smem) stage_begin(staged, c.image, bytes, &mbar);
-  // first tile of every warp: in flight while the image arrives
+  // Everything the kernel has to wait for before its first decision starts at once: the staging
+  // of `stage_bytes` (what the host planned for: the reserved room or the image buffer, whichever
+  // is smaller -- the bytes behind the live image are never looked at), the words the last rebuild
+  // published, the SLO mask, and every warp's first tile.
+  if (stage_bytes) stage_begin(staged, c.image, stage_bytes, &mbar);
+  const uint4 hdr = __ldg(reinterpret_cast<const uint4 *>(c.image_hdr));
+  const uint32_t slo_seen = __ldg(c.slo_seen);
   uint2 t4 = make_uint2(0, 0), a4 = make_uint2(0, 0);
   uint4 s4 = make_uint4(0, 0, 0, 0);
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -469,17 +473,18 @@ select_kernel(DeviceCatalog c, uint32_t image_smem, Queries q, uint64_t n, uint6
     s4 = __ldcs(reinterpret_cast<const uint4 *>(q.slo) + i4);
     a4 = __ldcs(reinterpret_cast<const uint2 *>(q.min_acc) + i4);
   }
-  if (in_smem) {
-    if (!stage_wait(&mbar)) {
-      if (threadIdx.x == 0) atomicMax(c.err, (uint32_t)DEV_ERR_STAGE_TIMEOUT);
-      return;
-    }
+  // the copy is waited for in any case: the CTA must not end with it in flight
+  if (stage_bytes && !stage_wait(&mbar)) {
+    if (threadIdx.x == 0) atomicMax(c.err, (uint32_t)DEV_ERR_STAGE_TIMEOUT);
+    return;
+  }
+  if (hdr.x <= stage_bytes) {
     SharedImage img{smem_u32(staged)};
-    select_body<Tally>(img, c, q, q0, span, park, t4, s4, a4);
+    select_body<Tally>(img, c, q, q0, span, park, hdr, slo_seen, t4, s4, a4);
   } else {
-    // the image does not fit in shared memory: read it from global memory (L1/L2 resident)
+    // the image is larger than what was staged: read it from global memory (L1/L2 resident)
     GlobalImage img{c.image};
-    select_body<Tally>(img, c, q, q0, span, park, t4, s4, a4);
+    select_body<Tally>(img, c, q, q0, span, park, hdr, slo_seen, t4, s4, a4);
   }
 }
 
@@ -512,10 +517,11 @@ cudaError_t launch_select(const DeviceCatalog &c, const uint16_t *d_task, const 
   grid = (n + per_cta - 1) / per_cta;
   if (grid > 0x7FFFFFFFull) return cudaErrorInvalidValue;
   Queries q{d_task, d_slo, d_min_acc, d_decision};
+  const uint32_t stage_bytes = (image_smem < c.image_capacity ? image_smem : c.image_capacity) & ~15u;
   if (tally)
-    select_kernel<true><<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n, per_cta);
+    select_kernel<true><<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, stage_bytes, q, n, per_cta);
   else
-    select_kernel<false><<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, image_smem, q, n, per_cta);
+    select_kernel<false><<<(uint32_t)grid, SELECT_THREADS, image_smem + PARK_BYTES, stream>>>(c, stage_bytes, q, n, per_cta);
   return cudaGetLastError();
 }
 
