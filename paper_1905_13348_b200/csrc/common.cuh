@@ -51,13 +51,13 @@ namespace infaas {
 // and nbw words), so the word an accuracy falls into does not depend on the task.
 //
 // Image (what the selection kernel stages in shared memory):
+//   dummy  64 bytes (what tasks without an index point at: every query of theirs reads
+//          "none" and goes to the slow path)
 //   hdr    (n_tasks + 1) u32, one per task: t2_off | (Ka + 1) << 24; entry n_tasks serves
 //          queries whose task is out of range; padded to 128 bytes
 //   rec    (n_tasks + 1) x SLO_BUCKETS u32 records, REC_STRIDE bytes apart
 //   bitmap (n_tasks + 1) x nbw u32: the accuracy bitmaps of the tasks' first segments,
 //          bitmap_stride(nbw) bytes apart
-//   dummy  64 bytes (what tasks without an index point at: every query of theirs reads
-//          "none" and goes to the slow path)
 //   var    per-segment blocks, each 16-byte aligned:
 //          ids   u32[F + 1] in REVERSE order: ids[p] sits at t2_off - 4 - 4p, and the slot
 //                of p = F holds PENDING -- the fast path needs no compare for "none"
@@ -88,21 +88,22 @@ inline __host__ __device__ uint32_t round_up_u32(uint32_t x, uint32_t a) { retur
 // shared-memory banks.
 constexpr uint32_t REC_STRIDE = 4u * (SLO_BUCKETS + 1u);   // bytes from one task's records to the next's
 inline __host__ __device__ uint32_t bitmap_stride(uint32_t nbw) { return 4u * (nbw | 1u); }   // same, bitmaps
-inline __host__ __device__ uint32_t image_rec_offset(uint32_t n_tasks) { return round_up_u32(4u * (n_tasks + 1u), 128u); }
+constexpr uint32_t IMAGE_DUMMY_BYTES = 64u;               // the dummy block opens the image
+constexpr uint32_t IMAGE_HDR_OFFSET = IMAGE_DUMMY_BYTES;  // the task words follow it
+inline __host__ __device__ uint32_t image_rec_offset(uint32_t n_tasks) {
+  return round_up_u32(IMAGE_HDR_OFFSET + 4u * (n_tasks + 1u), 128u);
+}
 inline __host__ __device__ uint32_t image_bitmap_offset(uint32_t n_tasks) {
   return image_rec_offset(n_tasks) + REC_STRIDE * (n_tasks + 1u);
 }
-inline __host__ __device__ uint32_t image_dummy_offset(uint32_t n_tasks, uint32_t nbw) {
+inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks, uint32_t nbw) {
   return round_up_u32(image_bitmap_offset(n_tasks) + bitmap_stride(nbw) * (n_tasks + 1u), 64u);
 }
-inline __host__ __device__ uint32_t image_var_offset(uint32_t n_tasks, uint32_t nbw) {
-  return image_dummy_offset(n_tasks, nbw) + 64u;
-}
-// The header word of a task without index (and of entry n_tasks): T2 is the one zero byte at
-// dummy + 16 with row width 0, the id slot of position 0 below it holds PENDING.
-inline __host__ __device__ uint32_t dummy_header(uint32_t n_tasks, uint32_t nbw) {
-  return image_dummy_offset(n_tasks, nbw) + 16u;
-}
+// The task word of a task without index (and of entry n_tasks): T2 is the one zero byte at
+// offset 16 of the dummy block with row width 0, the id slot of position 0 below it holds
+// PENDING.  The dummy block sits at the very start of the image, where the task word's 24-bit
+// offset reaches it however large the fixed tables are.
+constexpr uint32_t DUMMY_HEADER = 16u;
 
 // Byte offsets of the slow-path tables inside a segment's block, relative to their start
 // (8-byte aligned), for a list of F entries with Ks / Ka distinct latencies / accuracies.

@@ -144,7 +144,7 @@ template <bool Clamped, class Img>
 __device__ __forceinline__ uint32_t decide_fast(const Img &img, const Fixed &fx, uint32_t task, uint32_t slo,
                                                 uint32_t min_acc) {
   const uint32_t t = Clamped ? task : min(task, fx.n_tasks);
-  const uint32_t h = img.u32(t << 2);
+  const uint32_t h = img.u32(IMAGE_HDR_OFFSET + (t << 2));
   // bucket of the SLO: floor(bits(slo) * 2^-S) - bmin, saturated to 0..255 by the conversion
   const float code = __uint2float_rz(__float_as_uint(__uint2float_rz(slo)));
   uint32_t j;
@@ -240,7 +240,7 @@ __device__ __forceinline__ uint32_t decide_slow(const Img &img, const DeviceCata
   if (!(sl.z & TASK_FLAG_NOT_INDEXED)) {
     // the list's segments in order: the first has its header word and bitmap in the fixed part
     // of the image, the others (lists longer than INDEX_MAX_F) a header in global memory
-    const uint32_t h = img.u32(task << 2);
+    const uint32_t h = img.u32(IMAGE_HDR_OFFSET + (task << 2));
     uint32_t t2 = h & 0x00FFFFFFu, width = h >> 24, bm0 = fx.bm_off + task * fx.bm_stride;
     for (;;) {
       const uint32_t d = slow_segment(img, fx, sl, t2, width, bm0, slo, min_acc, best, best_p);

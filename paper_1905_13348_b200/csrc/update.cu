@@ -255,7 +255,7 @@ __device__ __forceinline__ void warp_prefix_count(const uint16_t *in, unsigned c
 // records and a bitmap that make every query of the task read "none".  All threads.
 __device__ __forceinline__ void write_dummy_task(const DeviceCatalog &c, uint32_t t) {
   const uint32_t T = c.n_tasks;
-  if (threadIdx.x == 0) reinterpret_cast<uint32_t *>(c.image)[t] = dummy_header(T, c.nbw);
+  if (threadIdx.x == 0) reinterpret_cast<uint32_t *>(c.image + IMAGE_HDR_OFFSET)[t] = DUMMY_HEADER;
   uint32_t *rec = reinterpret_cast<uint32_t *>(c.image + image_rec_offset(T) + t * REC_STRIDE);
   for (uint32_t j = threadIdx.x; j < SLO_BUCKETS; j += blockDim.x) rec[j] = 0u;
   uint32_t *bm = reinterpret_cast<uint32_t *>(c.image + image_bitmap_offset(T) + t * bitmap_stride(c.nbw));
@@ -521,7 +521,7 @@ __device__ bool build_index(const DeviceCatalog &c, uint32_t t, uint32_t F, Inde
   });
 
   if (tid == 0) {
-    if (first) reinterpret_cast<uint32_t *>(c.image)[t] = (base + BL.t2) | (width << 24);
+    if (first) reinterpret_cast<uint32_t *>(c.image + IMAGE_HDR_OFFSET)[t] = (base + BL.t2) | (width << 24);
     else c.xhdr[xi] = make_uint4(base + BL.t2, width, base + BL.bitmap, 0u);
     c.slow[first ? t : c.n_tasks + xi] = make_uint4(base + BL.slow, F | (Ks << 8) | (Ka << 16), 0u, Fs | (next << 8));
   }
@@ -829,9 +829,8 @@ rebuild_kernel(DeviceCatalog c, int advance, uint32_t window_us) {
   if (t == 0) {
     // entry n_tasks (queries whose task is out of range), the dummy block, and the bucket scale
     // every CTA has used, for the selection kernel
-    const uint32_t T = c.n_tasks, dummy = image_dummy_offset(T, c.nbw);
-    write_dummy_task(c, T);
-    if (tid < 16) reinterpret_cast<uint32_t *>(c.image + dummy)[tid] = tid == 3 ? PENDING : 0u;
+    write_dummy_task(c, c.n_tasks);
+    if (tid < IMAGE_DUMMY_BYTES / 4u) reinterpret_cast<uint32_t *>(c.image)[tid] = tid == 3 ? PENDING : 0u;
     if (tid == 0) {
       uint32_t Sh, bmin;
       bucket_scale(c, Sh, bmin);

@@ -329,6 +329,25 @@ def test_fused_window_call(name, kw, sizes):
         cat.free()
 
 
+@pytest.mark.parametrize("n_tasks,per_task", [(5000, 4), (20000, 3), (65535, 1)])
+def test_many_small_tasks(n_tasks, per_task):
+    """Thousands of tasks: the fixed tables of the index alone exceed shared memory (5000 tasks)
+    or even the range the task word's offset field addresses (20000 tasks: the tasks whose block
+    lies beyond it have no index and are answered by walking their lists).  Two windows with an
+    update between them."""
+    rng = np.random.default_rng(77)
+    nv = n_tasks * per_task
+    task = np.repeat(np.arange(n_tasks), per_task)
+    rows = rows_from(task, rng.choice(np.array([1, 2, 4, 8]), nv), rng.integers(500, 200_000, nv),
+                     rng.integers(5600, 8300, nv), rng.integers(1, 2000, nv), rng.integers(0, 3, nv))
+    rows = rows[rng.permutation(nv)]
+    n = 2 * 30_011
+    q_task = rng.integers(0, n_tasks + 2, n).astype(np.uint16)
+    q_slo = np.exp(rng.uniform(np.log(300.0), np.log(400_000.0), n)).astype(np.uint32)
+    q_acc = rng.integers(5000, 8600, n).astype(np.uint16)
+    run_both(W.Workload("many tasks", n_tasks, rows, q_task, q_slo, q_acc, 30_011, 20_000, "many small tasks"))
+
+
 def test_split_update_with_summed_counts_matches_whole_window():
     """infaas_tally / infaas_pending_counts / infaas_advance: two catalogs on this GPU stand
     in for two ranks; each decides its share of a window, the pending counts are summed and
