@@ -80,7 +80,7 @@ tally_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_varia
 // variants do not fit, the ids are split into `parts` ranges of `bins` ids: CTA b counts
 // range b % parts over the share b / parts of the decisions (every range sees all
 // decisions); the counters come from range 0 alone.
-constexpr int TALLY_SMEM_THREADS = 512;
+constexpr int TALLY_SMEM_THREADS = 1024;
 
 __global__ void __launch_bounds__(TALLY_SMEM_THREADS)
 tally_smem_kernel(const uint32_t *__restrict__ decision, uint64_t n, uint32_t n_variants, uint32_t bins,
@@ -854,9 +854,9 @@ cudaError_t launch_tally(const DeviceCatalog &c, const uint32_t *d_decision, uin
   if (n >= TALLY_SMEM_MIN_N && parts <= TALLY_SMEM_MAX_PARTS) {
     const uint32_t bins = ((c.n_variants + parts - 1) / parts + 3u) & ~3u;
     const size_t smem = (size_t)(bins + 32) * 4;                 // 32 spare bins
-    const uint32_t per_sm = smem > 100 * 1024 ? 1 : 2;
+    // one CTA of 1024 threads per SM: half as many histograms to clear and flush as two of 512
     uint64_t want = ((n >> 2) + TALLY_SMEM_THREADS * 8 - 1) / (TALLY_SMEM_THREADS * 8);
-    uint64_t shares = (uint64_t)sm_count * per_sm / parts;     // CTAs per id range
+    uint64_t shares = (uint64_t)sm_count / parts;              // CTAs per id range
     if (shares > want) shares = want;
     if (shares < 1) shares = 1;
     tally_smem_kernel<<<(uint32_t)(shares * parts), TALLY_SMEM_THREADS, smem, stream>>>(
